@@ -1,0 +1,170 @@
+/*
+ * vardrop.h -- C ABI of the B200 (sm_100a) implementation of VarDrop's per-batch training path
+ * (Kang et al., "VarDrop: Enhancing Training Efficiency by Reducing Variate Redundancy in Periodic Time
+ * Series Forecasting", AAAI-25).
+ *
+ * The path, in the order a training step calls it:
+ *   vardrop_hash      k-dominant frequency hashing of a batch (Algorithm 1)
+ *   vardrop_select    grouping by hash value and stratified sampling (Eq. 1, Eq. 2)
+ *   vardrop_attn_fwd  gather of the kept Q/K/V variate tokens + scaled dot-product attention (Eq. 3)
+ *   vardrop_attn_bwd  derivative of Eq. 3 over the kept tokens, gradients scattered to the full layout
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named in the argument lists are DEVICE pointers unless the comment says "host".
+ *     Configuration structs are host pointers and are read before the call returns.
+ *   - The caller owns every buffer, including the workspace `ws` (size from the matching
+ *     *_workspace_bytes query).  The library never allocates or frees device memory, never
+ *     synchronises the device and launches only on `stream` (a cudaStream_t passed as void*).
+ *   - Device pointers must be 16-byte aligned.
+ *   - The return value is a vardrop_status.  Problems found on the host (bad argument, unsupported
+ *     shape, short workspace, failed launch) are returned at once and nothing is launched.  Problems
+ *     found on the device (non-finite amplitude, a bounded wait that ran out) are written to the
+ *     first int32 of `ws` as a vardrop_status; read it with a device-to-host copy after
+ *     synchronising the stream.  vardrop_last_error() gives a thread-local text for the last non-OK return.
+ *   - Calls are thread-safe as long as concurrent calls use different workspaces.
+ */
+#ifndef VARDROP_H_
+#define VARDROP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    VARDROP_OK = 0,
+    VARDROP_ERR_INVALID_ARG = 1,   /* null/misaligned pointer, size out of range                       */
+    VARDROP_ERR_UNSUPPORTED = 2,   /* e.g. L with a prime factor above 7, head dimension other than 32/64 */
+    VARDROP_ERR_WORKSPACE = 3,     /* ws_bytes below the *_workspace_bytes answer                      */
+    VARDROP_ERR_CUDA = 4,          /* a CUDA runtime call or launch failed                             */
+    VARDROP_ERR_TIMEOUT = 5,       /* device side: a bounded wait gave up (device status word only)    */
+    VARDROP_ERR_NONFINITE = 6      /* device side: a candidate amplitude was NaN or infinite           */
+} vardrop_status;
+
+/* Static text for a status code; never freed. */
+const char* vardrop_status_string(int status);
+/* Thread-local detail of the last non-OK return on this thread ("" if none). */
+const char* vardrop_last_error(void);
+/* Library version, "major.minor". */
+const char* vardrop_version(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * k-dominant frequency hashing -- Algorithm 1 ("k-Dominant Frequency Hashing") and Definition 1.
+ *
+ *   step 1  amplitude spectrum A[b,n,f] = |sum_t x[b,n,t] exp(-2 pi i f t / L)| of every window
+ *   step 2  low-pass filter: only the bins f_lo <= f < f_hi are candidates
+ *   step 3  scope 0: mean over the batch, Abar[n,f] = (1/B) sum_b A[b,n,f]   (S = 1 hash row)
+ *           scope 1: every instance hashed on its own, Abar[b,n,f] = A[b,n,f] (S = B hash rows)
+ *   step 4  the k candidate bins of largest Abar in descending-amplitude order; equal amplitudes
+ *           rank the lower bin first
+ *   step 5  hash value = the ordered k-tuple packed 12 bits per bin, rank-1 bin most significant
+ *
+ * cfg (host)  B, N, L  shape of x;  1 <= k <= 5;  f_lo/f_hi candidate band, both 0 selects the default
+ *             f_lo = 1, f_hi = ceil((L/2+1)/2) (25 at L = 96, the cut-off of Appendix E);
+ *             requires 0 <= f_lo, f_lo + k <= f_hi <= L/2+1, f_hi <= 4096, L <= 8192 and L a product of 2, 3, 5, 7.
+ * x           [B, N, L] float32, contiguous.
+ * keys        [S, N] uint64 out.
+ * freqs       [S, N, k] int32 out, the ranked bins; may be NULL.
+ * amp_dbg     [S, N, f_hi - f_lo] float32 out, Abar; may be NULL.
+ * ws          no scratch is used beyond the status word; pass at least vardrop_hash_workspace_bytes.
+ * Device status: VARDROP_ERR_NONFINITE when a candidate amplitude is not finite (keys then unspecified).
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t B, N, L, k;
+    int32_t f_lo, f_hi;
+    int32_t scope;
+} vardrop_hash_cfg;
+
+size_t vardrop_hash_workspace_bytes(const vardrop_hash_cfg* cfg);
+int vardrop_hash(const float* x, const vardrop_hash_cfg* cfg, uint64_t* keys, int32_t* freqs, float* amp_dbg,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Grouping and stratified sampling -- last sentence of "Procedure of k-DFH" (variates with the same
+ * hash value form a group), Eq. 1 (|S_i| = min(|G_i|, gs)), Eq. 2 (S = union of the S_i), and the
+ * token reduction ratio delta = 1 - n_sel / N of Sec. 3.3.
+ *
+ * Per hash row s (S rows, independent):
+ *   groups    classes of equal key; group ids are dense ranks in ascending key order; members of a
+ *             group are ordered by ascending variate index
+ *   quota     q_g = min(|G_g|, gs if gs > 0, max(1, ceil(|G_g| * rate_ppm / 10^6))), rate_ppm =
+ *             round(rate * 10^6), integer arithmetic; rate = 1 is Eq. 1 itself
+ *   sampling  member j of group g gets priority = word 0 of Philox4x32-10(counter (j, g, s, step),
+ *             key (seed low, seed high)); the q_g members of smallest (priority, j) are kept
+ *
+ * cfg (host)    S, N (1 <= N <= 65536), gs (<= 0: no cap), rate in (0, 1], seed, step.
+ * keys          [S, N] uint64 in.
+ * group_id      [S, N] int32 out.
+ * group_offsets [S, N+1] int32 out; entry g is the start of group g in `members`, entries past the
+ *               number of groups equal N.
+ * members       [S, N] int32 out; variates sorted by (key, index).
+ * n_groups      [S] int32 out.
+ * sel_idx       [S, N] int32 out; kept variates ascending, first n_sel[s] valid, the rest -1.
+ * n_sel         [S] int32 out.
+ * inv_idx       [S, N] int32 out; position of variate n in sel_idx, or -1 when dropped.
+ * ws            scratch of vardrop_select_workspace_bytes; contents are scratch only.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t S, N, gs;
+    double rate;
+    uint64_t seed;
+    uint32_t step;
+} vardrop_select_cfg;
+
+size_t vardrop_select_workspace_bytes(const vardrop_select_cfg* cfg);
+int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t* group_id, int32_t* group_offsets,
+                   int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Attention over the kept tokens -- Sec. 3.3 (token reduction: only the selected variate tokens enter
+ * self-attention) and Eq. 3, per batch instance b and head h:
+ *   Q' = q[b, sel_idx[0..n_sel), h, :] (same for K', V');  O' = softmax(Q' K'^T * sm_scale) V';
+ *   lse_i = log sum_j exp(S_ij).
+ * bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before the second product.
+ *
+ * cfg (host)  B, N, H, D (D = 32 or 64; N <= 65536), sm_scale (0 selects 1/sqrt(D)).
+ * q, k, v     [B, N, H, D] bf16, contiguous.
+ * sel_idx     [N] int32, ascending kept variates (row 0 of vardrop_select's output), or NULL for the
+ *             all-token path (VarDrop off, the inference / "ground" configuration of the paper).
+ * n_sel       [1] int32 on the device, number of valid entries of sel_idx; ignored when sel_idx is NULL.
+ * o           [B, N, H, D] bf16 out; rows 0..n_sel-1 of every instance hold O', the rest is untouched.
+ * lse         [B, H, N] float32 out; entries 0..n_sel-1 valid.
+ * ws          scratch of vardrop_attn_workspace_bytes.  After the call it holds the gathered Q', K', V';
+ *             vardrop_attn_bwd for the same step must be given the same, unmodified workspace.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t B, N, H, D;
+    float sm_scale;
+} vardrop_attn_cfg;
+
+size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg);
+int vardrop_attn_fwd(const void* q, const void* k, const void* v, const int32_t* sel_idx, const int32_t* n_sel,
+                     const vardrop_attn_cfg* cfg, void* o, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Backward of the above (the paper applies VarDrop in training only, Sec. 3.1; the derivative of
+ * Eq. 3 is the chain rule):
+ *   dV' = P^T dO';  dP = dO' V'^T;  Delta_i = sum_d dO'_id O'_id;  dS = P o (dP - Delta);
+ *   dQ' = dS K' sm_scale;  dK' = dS^T Q' sm_scale,
+ * then scattered: row sel_idx[i] of dq/dk/dv receives row i of dQ'/dK'/dV'; rows of dropped variates
+ * are written as zeros, so every row of dq, dk, dv is written exactly once.
+ *
+ * q, k, v, sel_idx, n_sel, cfg, ws   as given to vardrop_attn_fwd (ws unmodified since).
+ * o, lse      outputs of vardrop_attn_fwd.
+ * d_o         [B, N, H, D] bf16, gradient of o; rows 0..n_sel-1 are read.
+ * inv_idx     [N] int32 from vardrop_select (NULL when sel_idx is NULL).
+ * dq, dk, dv  [B, N, H, D] bf16 out, full variate layout.
+ * dQ' is accumulated across key tiles with fp32 atomic adds, so its low-order bits may differ from run
+ * to run; dK', dV' are bit-reproducible.
+ * ---------------------------------------------------------------------------------------------- */
+int vardrop_attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                     const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg* cfg,
+                     void* dq, void* dk, void* dv, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VARDROP_H_ */

@@ -1,0 +1,396 @@
+// Attention backward over the kept variate tokens and the scatter of the gradients to the full layout.
+//
+// bwd_prep_kernel    Delta_i = sum_d dO'_id O'_id, a zero-filled staged copy of dO' (rows past n_sel may hold
+//                    anything in the caller's buffer), and the zeroing of the fp32 dQ' accumulator.
+// attn_bwd_kernel    one CTA per (128-key tile, head, instance) looping over the query tiles.  Scores are
+//                    formed transposed (S^T = K Q^T, dP^T = V dO^T) so that each of the 128 threads owns one key
+//                    row of tensor memory; P^T and dS^T are written to shared memory once and feed three
+//                    tensor-core products: dV += P^T dO, dK += dS^T Q (accumulated in tensor memory across the
+//                    query loop) and dQ_i = dS K (added into the fp32 accumulator with atomics).
+// bwd_finish_kernel  dq rows from the accumulator (scaled, bf16) and zero rows for every dropped variate, so
+//                    each row of dq / dk / dv is written exactly once.
+#include "attn_common.cuh"
+
+namespace vardrop {
+
+namespace {
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ float2 unpack2(uint32_t w) {
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w));
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// prep
+// ---------------------------------------------------------------------------------------------------------
+struct PrepParams {
+    const uint4* o;       // [B, N, H, D] bf16
+    const uint4* d_o;     // [B, N, H, D] bf16
+    uint4* dog;           // [B, Ncap, H, 64] bf16 staged dO (NULL: not needed)
+    float* delta;         // [B, H, Ncap]
+    float4* dq_acc;       // [B, Ncap, H, 64] fp32
+    const int32_t* n_sel; // NULL: N
+    int N, Ncap, H, D;
+};
+
+// one thread per 16-byte chunk of a staged (token, head) row; the 8 threads of a row reduce Delta by shuffles
+__global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
+    const int n_sel = P.n_sel ? *P.n_sel : P.N;
+    const int n_fill = min(P.Ncap, (n_sel + kTile - 1) / kTile * kTile);
+    const int b = blockIdx.y;
+    const int chunks_row = P.H * 8;
+    const int src_chunks_head = P.D / 8;
+    const int total = n_fill * chunks_row;            // a multiple of 8; blockDim is a multiple of 8
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int i = idx / chunks_row;
+        const int c = idx - i * chunks_row;
+        const int h = c >> 3, dc = c & 7;
+        uint4 vo = make_uint4(0u, 0u, 0u, 0u), vd = vo;
+        if (i < n_sel && dc < src_chunks_head) {
+            const size_t src = (static_cast<size_t>(b) * P.N + i) * (P.H * src_chunks_head) + h * src_chunks_head + dc;
+            vo = __ldg(P.o + src);
+            vd = __ldg(P.d_o + src);
+        }
+        const float2 a0 = unpack2(vo.x), a1 = unpack2(vo.y), a2 = unpack2(vo.z), a3 = unpack2(vo.w);
+        const float2 g0 = unpack2(vd.x), g1 = unpack2(vd.y), g2 = unpack2(vd.z), g3 = unpack2(vd.w);
+        float part = a0.x * g0.x + a0.y * g0.y + a1.x * g1.x + a1.y * g1.y + a2.x * g2.x + a2.y * g2.y + a3.x * g3.x + a3.y * g3.y;
+        part += __shfl_xor_sync(0xffffffffu, part, 1);
+        part += __shfl_xor_sync(0xffffffffu, part, 2);
+        part += __shfl_xor_sync(0xffffffffu, part, 4);
+        if (dc == 0) P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + i] = part;
+        const size_t dst = (static_cast<size_t>(b) * P.Ncap + i) * chunks_row + c;
+        if (P.dog) P.dog[dst] = vd;
+        P.dq_acc[2 * dst] = make_float4(0.f, 0.f, 0.f, 0.f);
+        P.dq_acc[2 * dst + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// main
+// ---------------------------------------------------------------------------------------------------------
+struct BwdParams {
+    const float* lse;       // [B, H, N]
+    const float* delta;     // [B, H, Ncap]
+    float* dq_acc;          // [B, Ncap, H, 64]
+    __nv_bfloat16* dk;      // [B, N, H, D]
+    __nv_bfloat16* dv;
+    const int32_t* sel_idx; // NULL: identity
+    const int32_t* n_sel;   // NULL: N
+    int* status;
+    int N, Ncap, H, D;
+    float scale, scale_log2;
+};
+
+constexpr int kBwdThreads = 128;
+constexpr uint32_t kBwdTmemCols = 512;
+constexpr int kBwdSmemBytes = 2048 /*barriers, row statistics, alignment*/ + 4 * kTileBytes /*K, V, Q, dO*/ + 4 * kTileBytes /*P^T, dS^T*/;
+
+// 32 consecutive columns of row r of a 128 x 128 bf16 tile stored as two 64-column panels (128-byte swizzled rows)
+__device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0, const float* v) {
+    unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
+    const int chunk0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint4 w = make_uint4(pack2(v[8 * q + 0], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                   pack2(v[8 * q + 6], v[8 * q + 7]));
+        *reinterpret_cast<uint4*>(panel + (((chunk0 + q) ^ (r & 7)) << 4)) = w;
+    }
+}
+
+__global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                const __grid_constant__ CUtensorMap map_k,
+                                                                const __grid_constant__ CUtensorMap map_v,
+                                                                const __grid_constant__ CUtensorMap map_do, const BwdParams P) {
+    const int n_sel = P.n_sel ? *P.n_sel : P.N;
+    const int jt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    if (jt * kTile >= n_sel) return;
+    const int n_q = (n_sel + kTile - 1) / kTile;
+
+    extern __shared__ unsigned char smem_dyn[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
+    uint64_t* bar_kv = bars + 0;
+    uint64_t* bar_qdo = bars + 1;
+    uint64_t* bar_s = bars + 2;
+    uint64_t* bar_g = bars + 3;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
+    float* s_lse = reinterpret_cast<float*>(smem_dyn + 64);       // [128] log2-domain row statistics of the query tile
+    float* s_delta = s_lse + kTile;                               // [128]
+    unsigned char* sK = align_tiles(smem_dyn + 64 + 2 * kTile * sizeof(float));
+    unsigned char* sV = sK + kTileBytes;
+    unsigned char* sQ = sV + kTileBytes;
+    unsigned char* sdO = sQ + kTileBytes;
+    unsigned char* sPt = sdO + kTileBytes;          // P^T  : rows = keys, columns = queries (two 64-query panels)
+    unsigned char* sdSt = sPt + 2 * kTileBytes;     // dS^T : same shape
+    if (sdSt + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
+        if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
+        return;
+    }
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, kBwdTmemCols);
+        tmem_relinquish();
+    }
+    if (tid == 0) {
+        mbar_init(bar_kv, 1);
+        mbar_init(bar_qdo, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_g, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+        tma_prefetch_desc(&map_do);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tm_st = tmem;            // [0,128)   S^T
+    const uint32_t tm_dpt = tmem + 128;     // [128,256) dP^T
+    const uint32_t tm_dv = tmem + 256;      // [256,320) dV
+    const uint32_t tm_dk = tmem + 320;      // [320,384) dK
+    const uint32_t tm_dq = tmem + 384;      // [384,448) dQ of the current query tile
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+
+    constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);     // K-major x K-major, N = 128
+    constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major, B MN-major, N = 64
+    constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_kv, 2 * kTileBytes);
+        tma_load_4d(sK, &map_k, bar_kv, 0, h, jt * kTile, b);
+        tma_load_4d(sV, &map_v, bar_kv, 0, h, jt * kTile, b);
+    }
+    const int key = jt * kTile + tid;               // this thread's key row
+    const bool key_valid = key < n_sel;
+    bool ok = true;
+
+    for (int i = 0; i < n_q; ++i) {
+        if (tid == 0) {                              // sQ / sdO were released by the wait on bar_g of tile i-1
+            mbar_expect_tx(bar_qdo, 2 * kTileBytes);
+            tma_load_4d(sQ, &map_q, bar_qdo, 0, h, i * kTile, b);
+            tma_load_4d(sdO, &map_do, bar_qdo, 0, h, i * kTile, b);
+        }
+        {
+            const int qrow = i * kTile + tid;
+            const bool qv = qrow < n_sel;
+            s_lse[tid] = qv ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
+            s_delta[tid] = qv ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
+        }
+        if (tid == 0) {
+            if (i == 0) ok &= mbar_wait(bar_kv, 0);
+            ok &= mbar_wait(bar_qdo, i & 1);
+            tc_fence_after();
+            const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ), d0 = smem_u32(sdO);
+#pragma unroll
+            for (int ks = 0; ks < kDP / 16; ++ks)
+                tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < kDP / 16; ++ks)
+                tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+            tc_commit(bar_s);
+        }
+        __syncthreads();                             // row statistics visible
+        ok &= mbar_wait(bar_s, i & 1);
+        tc_fence_after();
+
+        // ---- P^T and dS^T of this thread's key row over the 128 queries of the tile --------------------------
+        float sv[32], dp[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tm_st + lane_sel + c * 32, sv);
+            tmem_ld32(tm_dpt + lane_sel + c * 32, dp);
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                const int col = c * 32 + x;
+                const float p = key_valid ? exp2f(fmaf(sv[x], P.scale_log2, -s_lse[col])) : 0.f;
+                sv[x] = p;
+                dp[x] = p * (dp[x] - s_delta[col]);
+            }
+            store_chunk32(sPt, tid, c * 32, sv);
+            store_chunk32(sdSt, tid, c * 32, dp);
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ), d0 = smem_u32(sdO), k0 = smem_u32(sK);
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
+                const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
+                tc_mma_bf16(tm_dv, umma_desc_sw128(pt + a_off, 16, 1024), umma_desc_sw128(d0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
+                            (i > 0) | (ks > 0));
+                tc_mma_bf16(tm_dk, umma_desc_sw128(dst + a_off, 16, 1024), umma_desc_sw128(q0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
+                            (i > 0) | (ks > 0));
+            }
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K
+                tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
+                            idesc_mnmn, ks > 0);
+            tc_commit(bar_g);
+        }
+        ok &= mbar_wait(bar_g, i & 1);
+        tc_fence_after();
+        {
+            const int qrow = i * kTile + tid;        // tensor-memory lane = query row of dQ_i
+            float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP;
+#pragma unroll
+            for (int c = 0; c < kDP / 32; ++c) {
+                tmem_ld32(tm_dq + lane_sel + c * 32, sv);
+                tmem_ld_wait();
+                if (qrow < n_sel) {
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) atomicAdd(dst + c * 32 + x, sv[x]);
+                }
+            }
+        }
+        tc_fence_before();
+        if (!__syncthreads_and(ok)) break;
+    }
+
+    if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
+    {   // tensor-memory loads are warp-collective: every thread takes part, only valid key rows store
+        const bool store = ok && key_valid;
+        const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
+        const size_t row = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
+        float acc[32];
+#pragma unroll
+        for (int c = 0; c < kDP / 32; ++c) {
+            if (c * 32 < P.D) {
+                tmem_ld32(tm_dv + lane_sel + c * 32, acc);
+                tmem_ld_wait();
+                if (store) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4*>(P.dv + row + c * 32 + q * 8) =
+                            make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
+                                       pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
+                }
+                tmem_ld32(tm_dk + lane_sel + c * 32, acc);
+                tmem_ld_wait();
+                if (store) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4*>(P.dk + row + c * 32 + q * 8) =
+                            make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
+                                       pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// finish
+// ---------------------------------------------------------------------------------------------------------
+struct FinishParams {
+    const float4* dq_acc;    // [B, Ncap, H, 64] fp32
+    uint4 *dq, *dk, *dv;     // [B, N, H, D] bf16
+    const int32_t* inv_idx;  // NULL: identity
+    int N, Ncap, H, D;
+    float scale;
+};
+
+__global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
+    const int b = blockIdx.y;
+    const int chunks_head = P.D / 8;
+    const int chunks_row = P.H * chunks_head;
+    const int total = P.N * chunks_row;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int n = idx / chunks_row;
+        const int c = idx - n * chunks_row;
+        const int h = c / chunks_head, dc = c - h * chunks_head;
+        const int j = P.inv_idx ? P.inv_idx[n] : n;
+        const size_t dst = static_cast<size_t>(b) * total + idx;
+        if (j >= 0) {
+            const float4* src = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * (kDP / 4) + dc * 2;
+            const float4 a = __ldcg(src), c2 = __ldcg(src + 1);
+            P.dq[dst] = make_uint4(pack2(a.x * P.scale, a.y * P.scale), pack2(a.z * P.scale, a.w * P.scale),
+                                   pack2(c2.x * P.scale, c2.y * P.scale), pack2(c2.z * P.scale, c2.w * P.scale));
+        } else {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            P.dq[dst] = z;
+            P.dk[dst] = z;
+            P.dv[dst] = z;
+        }
+    }
+}
+
+}  // namespace
+
+int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                    const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg& c, void* dq,
+                    void* dk, void* dv, void* ws, cudaStream_t stream) {
+    const AttnWs w = attn_layout(c);
+    char* base = static_cast<char*>(ws);
+    const bool staged = attn_uses_staging(c, sel_idx);
+    const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
+
+    PrepParams R{};
+    R.o = static_cast<const uint4*>(o); R.d_o = static_cast<const uint4*>(d_o);
+    R.dog = staged ? reinterpret_cast<uint4*>(base + w.dog) : nullptr;
+    R.delta = reinterpret_cast<float*>(base + w.delta);
+    R.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
+    R.n_sel = sel_idx ? n_sel : nullptr;
+    R.N = c.N; R.Ncap = w.Ncap; R.H = c.H; R.D = c.D;
+    {
+        const long long work = static_cast<long long>(w.Ncap) * c.H * 8;
+        int gx = static_cast<int>((work + 255) / 256);
+        if (gx > 1184) gx = 1184;
+        bwd_prep_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(R);
+        if (int st = check_cuda(cudaGetLastError(), "attention: backward prep launch")) return st;
+    }
+
+    CUtensorMap mq, mk, mv, mdo;
+    if (staged) {
+        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mdo, base + w.dog, c.B, w.Ncap, w.Ncap, c.H)) return st;
+    } else {
+        if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mv, v, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mdo, d_o, c.B, c.N, c.N, c.H)) return st;
+    }
+    BwdParams P{};
+    P.lse = lse; P.delta = R.delta; P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
+    P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
+    P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
+    P.status = reinterpret_cast<int*>(base);
+    P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
+    P.scale = scale; P.scale_log2 = scale * 1.4426950408889634f;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_dev != dev) {
+        if (int st = check_cuda(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemBytes), "attention: smem attribute")) return st;
+        attr_dev = dev;
+    }
+    attn_bwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P);
+    if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
+
+    FinishParams F{};
+    F.dq_acc = reinterpret_cast<const float4*>(base + w.dq_acc);
+    F.dq = static_cast<uint4*>(dq); F.dk = static_cast<uint4*>(dk); F.dv = static_cast<uint4*>(dv);
+    F.inv_idx = sel_idx ? inv_idx : nullptr;
+    F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.scale = scale;
+    {
+        const long long work = static_cast<long long>(c.N) * c.H * (c.D / 8);
+        int gx = static_cast<int>((work + 255) / 256);
+        if (gx > 1184) gx = 1184;
+        bwd_finish_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F);
+    }
+    return check_cuda(cudaGetLastError(), "attention: backward finish launch");
+}
+
+}  // namespace vardrop

@@ -1,0 +1,336 @@
+// Token gather and attention forward (Eq. 3) over the kept variate tokens.
+//
+// gather_kernel     compacts q/k/v rows named by sel_idx into [B, Ncap, H, 64] staging buffers with 16-byte
+//                   copies, zero-pads D = 32 to 64 and zero-fills the ragged end of the last 128-token tile.
+// attn_fwd_kernel   one CTA per (128-query tile, head, instance): TMA loads the Q tile once and streams K/V
+//                   tiles through a two-stage ring; S = Q K^T and O_j = P V run on the tcgen05 tensor cores
+//                   with accumulators in tensor memory; the online softmax is done by 128 threads, one
+//                   query row each, straight from tensor memory.
+#include "attn_common.cuh"
+
+namespace vardrop {
+
+// ---------------------------------------------------------------------------------------------------------
+// host: tensor maps
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int token_stride, int H) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(kDP), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(tokens),
+                                static_cast<cuuint64_t>(B)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kRowBytes), static_cast<cuuint64_t>(H) * kRowBytes,
+                                   static_cast<cuuint64_t>(token_stride) * H * kRowBytes};
+    const cuuint32_t box[4] = {kDP, 1, kTile, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r));
+    return VARDROP_OK;
+}
+
+int attn_validate(const vardrop_attn_cfg& c) {
+    if (c.B < 1 || c.N < 1 || c.H < 1) return fail(VARDROP_ERR_INVALID_ARG, "attention: B, N, H >= 1 required (B=%d N=%d H=%d)", c.B, c.N, c.H);
+    if (c.D != 32 && c.D != 64) return fail(VARDROP_ERR_UNSUPPORTED, "attention: head dimension %d (32 or 64 supported)", c.D);
+    if (c.N > 65536) return fail(VARDROP_ERR_UNSUPPORTED, "attention: N=%d above 65536", c.N);
+    if (c.H > 65535 || c.B > 65535) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B or H above 65535");
+    if (!(c.sm_scale >= 0.f)) return fail(VARDROP_ERR_INVALID_ARG, "attention: sm_scale must be >= 0 (0 selects 1/sqrt(D))");
+    return VARDROP_OK;
+}
+
+size_t attn_workspace_bytes(const vardrop_attn_cfg& c) { return attn_layout(c).total; }
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------------------
+// gather
+// ---------------------------------------------------------------------------------------------------------
+struct GatherParams {
+    const uint4* src[3];
+    uint4* dst[3];
+    const int32_t* sel_idx;   // NULL: identity
+    const int32_t* n_sel;     // NULL with sel_idx NULL
+    int N, Ncap, H, D;
+};
+
+__global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
+    const int n_sel = P.sel_idx ? *P.n_sel : P.N;
+    const int n_fill = min(P.Ncap, (n_sel + kTile - 1) / kTile * kTile);     // rows to define: kept + zero tail of the tile
+    const int chunks_row = P.H * (kDP / 8);                                   // 16-byte chunks per staged token
+    const int src_chunks_head = P.D / 8;
+    const int b = blockIdx.y, t = blockIdx.z;
+    const int total = n_fill * chunks_row;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int j = idx / chunks_row;
+        const int c = idx - j * chunks_row;
+        const int h = c / (kDP / 8), dc = c - h * (kDP / 8);
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (j < n_sel && dc < src_chunks_head) {
+            const int n = P.sel_idx ? P.sel_idx[j] : j;
+            val = __ldg(P.src[t] + (static_cast<size_t>(b) * P.N + n) * (P.H * src_chunks_head) + h * src_chunks_head + dc);
+        }
+        P.dst[t][(static_cast<size_t>(b) * P.Ncap + j) * chunks_row + c] = val;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// forward
+// ---------------------------------------------------------------------------------------------------------
+struct FwdParams {
+    __nv_bfloat16* o;
+    float* lse;
+    const int32_t* n_sel;   // NULL: all N tokens
+    int* status;
+    int N, H, D;
+    float scale_log2;       // sm_scale * log2(e)
+};
+
+constexpr int kFwdThreads = 128;
+constexpr uint32_t kFwdTmemCols = 256;
+constexpr int kFwdSmemBytes = 1024 /*barriers + alignment*/ + kTileBytes /*Q*/ + 2 * kTileBytes /*K*/ + 2 * kTileBytes /*V*/ + 2 * kTileBytes /*P*/;
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Writes 32 consecutive columns (c0 .. c0+31, c0 a multiple of 32) of row `r` of a 128 x 128 bf16 tile held as two
+// K-major panels of 64 columns, each row 128 bytes with the 128-byte swizzle.
+__device__ __forceinline__ void store_row_chunk32(unsigned char* tile, int r, int c0, const float* v) {
+    unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
+    const int chunk0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint4 w = make_uint4(pack_bf16(v[8 * q + 0], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                                   pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+        *reinterpret_cast<uint4*>(panel + (((chunk0 + q) ^ (r & 7)) << 4)) = w;
+    }
+}
+
+__global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                const __grid_constant__ CUtensorMap map_k,
+                                                                const __grid_constant__ CUtensorMap map_v, const FwdParams P) {
+    const int n_sel = P.n_sel ? *P.n_sel : P.N;
+    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    if (qt * kTile >= n_sel) return;
+    const int n_kv = (n_sel + kTile - 1) / kTile;
+
+    extern __shared__ unsigned char smem_dyn[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);     // barriers and the TMEM slot sit in front of the tiles
+    uint64_t* bar_q = bars + 0;
+    uint64_t* bar_kv = bars + 1;                    // [2]
+    uint64_t* bar_s = bars + 3;
+    uint64_t* bar_o = bars + 4;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+    unsigned char* sQ = align_tiles(smem_dyn + 64);
+    unsigned char* sK = sQ + kTileBytes;            // 2 stages
+    unsigned char* sV = sK + 2 * kTileBytes;        // 2 stages
+    unsigned char* sP = sV + 2 * kTileBytes;        // 128 x 128 bf16, two K-major panels
+    if (sP + 2 * kTileBytes > smem_dyn + kFwdSmemBytes) {       // dynamic shared memory base not 1024-byte aligned
+        if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
+        return;
+    }
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, kFwdTmemCols);
+        tmem_relinquish();
+    }
+    if (tid == 0) {
+        mbar_init(bar_q, 1);
+        mbar_init(bar_kv + 0, 1);
+        mbar_init(bar_kv + 1, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tmem_s = tmem;                   // columns [0, 128): S
+    const uint32_t tmem_o = tmem + 128;             // columns [128, 192): P V of the current key tile
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+
+    constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
+    constexpr uint32_t idesc_o = umma_idesc_bf16(128, kDP, 0, 1);
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_q, kTileBytes);
+        tma_load_4d(sQ, &map_q, bar_q, 0, h, qt * kTile, b);
+        mbar_expect_tx(bar_kv, 2 * kTileBytes);
+        tma_load_4d(sK, &map_k, bar_kv, 0, h, 0, b);
+        tma_load_4d(sV, &map_v, bar_kv, 0, h, 0, b);
+    }
+
+    float o_acc[kDP];
+#pragma unroll
+    for (int d = 0; d < kDP; ++d) o_acc[d] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+
+    for (int j = 0; j < n_kv; ++j) {
+        const int st = j & 1;
+        if (tid == 0) {
+            if (j + 1 < n_kv) {                      // the other stage was released by the wait on bar_o of tile j-1
+                mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
+                tma_load_4d(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
+                tma_load_4d(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
+            }
+            if (j == 0) ok &= mbar_wait(bar_q, 0);
+            ok &= mbar_wait(bar_kv + st, (j >> 1) & 1);
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(sK + st * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kDP / 16; ++ks)
+                tc_mma_bf16(tmem_s, umma_desc_sw128(a0 + ks * 32, 16, 1024), umma_desc_sw128(b0 + ks * 32, 16, 1024), idesc_s, ks > 0);
+            tc_commit(bar_s);
+        }
+        ok &= mbar_wait(bar_s, j & 1);
+        tc_fence_after();
+
+        // ---- online softmax of this thread's query row over the 128 keys of the tile ----------------------
+        const int valid = min(kTile, n_sel - j * kTile);      // keys of this tile that exist
+        float s[32];
+        float m_tile = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_s + lane_sel + c * 32, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (c * 32 + i < valid) m_tile = fmaxf(m_tile, s[i]);
+        }
+        const float m_new = fmaxf(m_run, m_tile * P.scale_log2);
+        const float alpha = exp2f(m_run - m_new);
+        float l_tile = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_s + lane_sel + c * 32, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float p = (c * 32 + i < valid) ? exp2f(fmaf(s[i], P.scale_log2, -m_new)) : 0.f;
+                s[i] = p;
+                l_tile += p;
+            }
+            store_row_chunk32(sP, tid, c * 32, s);
+        }
+        l_run = l_run * alpha + l_tile;
+        m_run = m_new;
+#pragma unroll
+        for (int d = 0; d < kDP; ++d) o_acc[d] *= alpha;
+
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(sP), b0 = smem_u32(sV + st * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks)
+                tc_mma_bf16(tmem_o, umma_desc_sw128(a0 + (ks >> 2) * kTileBytes + (ks & 3) * 32, 16, 1024),
+                            umma_desc_sw128(b0 + ks * 2048, kTileBytes, 1024), idesc_o, ks > 0);
+            tc_commit(bar_o);
+        }
+        ok &= mbar_wait(bar_o, j & 1);
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < kDP / 32; ++c) {
+            tmem_ld32(tmem_o + lane_sel + c * 32, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o_acc[c * 32 + i] += s[i];
+        }
+        tc_fence_before();
+        if (!__syncthreads_and(ok)) break;           // a wait gave up somewhere in the CTA: stop issuing work
+    }
+
+    if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
+    const int row = qt * kTile + tid;
+    if (ok && row < n_sel) {
+        const float inv_l = 1.f / l_run;
+        __nv_bfloat16* dst = P.o + ((static_cast<size_t>(b) * P.N + row) * P.H + h) * P.D;
+#pragma unroll
+        for (int q = 0; q < kDP / 8; ++q) {
+            if (q * 8 < P.D) {
+                const uint4 w = make_uint4(pack_bf16(o_acc[8 * q + 0] * inv_l, o_acc[8 * q + 1] * inv_l),
+                                           pack_bf16(o_acc[8 * q + 2] * inv_l, o_acc[8 * q + 3] * inv_l),
+                                           pack_bf16(o_acc[8 * q + 4] * inv_l, o_acc[8 * q + 5] * inv_l),
+                                           pack_bf16(o_acc[8 * q + 6] * inv_l, o_acc[8 * q + 7] * inv_l));
+                *reinterpret_cast<uint4*>(dst + 8 * q) = w;
+            }
+        }
+        P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kFwdTmemCols);
+}
+
+}  // namespace
+
+int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* sel_idx, const int32_t* n_sel,
+                    const vardrop_attn_cfg& c, void* o, float* lse, void* ws, cudaStream_t stream) {
+    const AttnWs w = attn_layout(c);
+    char* base = static_cast<char*>(ws);
+    if (int st = check_cuda(cudaMemsetAsync(ws, 0, sizeof(int), stream), "attention: clear status")) return st;
+    const bool staged = attn_uses_staging(c, sel_idx);
+    CUtensorMap mq, mk, mv;
+    if (staged) {
+        GatherParams G{};
+        G.src[0] = static_cast<const uint4*>(q); G.src[1] = static_cast<const uint4*>(k); G.src[2] = static_cast<const uint4*>(v);
+        G.dst[0] = reinterpret_cast<uint4*>(base + w.qg); G.dst[1] = reinterpret_cast<uint4*>(base + w.kg);
+        G.dst[2] = reinterpret_cast<uint4*>(base + w.vg);
+        G.sel_idx = sel_idx; G.n_sel = sel_idx ? n_sel : nullptr;
+        G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D;
+        const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
+        int gx = static_cast<int>((work + 255) / 256);
+        if (gx > 1184) gx = 1184;
+        gather_kernel<<<dim3(gx, c.B, 3), 256, 0, stream>>>(G);
+        if (int st = check_cuda(cudaGetLastError(), "attention: gather launch")) return st;
+        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+    } else {
+        if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mv, v, c.B, c.N, c.N, c.H)) return st;
+    }
+    FwdParams P{};
+    P.o = static_cast<__nv_bfloat16*>(o); P.lse = lse; P.n_sel = sel_idx ? n_sel : nullptr;
+    P.status = reinterpret_cast<int*>(base);
+    P.N = c.N; P.H = c.H; P.D = c.D;
+    const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
+    P.scale_log2 = scale * 1.4426950408889634f;
+    static thread_local int attr_dev = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_dev != dev) {
+        if (int st = check_cuda(cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmemBytes), "attention: smem attribute")) return st;
+        attr_dev = dev;
+    }
+    attn_fwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P);
+    return check_cuda(cudaGetLastError(), "attention: forward launch");
+}
+
+}  // namespace vardrop

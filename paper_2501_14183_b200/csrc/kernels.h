@@ -1,0 +1,33 @@
+// Internal launch interface between the C-ABI layer and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/vardrop.h"
+
+namespace vardrop {
+
+// hash.cu
+size_t hash_workspace_bytes(const vardrop_hash_cfg& cfg);
+int hash_validate(const vardrop_hash_cfg& cfg, int* f_lo, int* f_hi);
+int hash_launch(const float* x, const vardrop_hash_cfg& cfg, uint64_t* keys, int32_t* freqs, float* amp_dbg, int* status,
+                cudaStream_t stream);
+
+// select.cu
+size_t select_workspace_bytes(const vardrop_select_cfg& cfg);
+int select_validate(const vardrop_select_cfg& cfg);
+int select_launch(const uint64_t* keys, const vardrop_select_cfg& cfg, int32_t* group_id, int32_t* group_offsets, int32_t* members,
+                  int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, void* ws, cudaStream_t stream);
+
+// attn_*.cu
+size_t attn_workspace_bytes(const vardrop_attn_cfg& cfg);
+int attn_validate(const vardrop_attn_cfg& cfg);
+int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* sel_idx, const int32_t* n_sel,
+                    const vardrop_attn_cfg& cfg, void* o, float* lse, void* ws, cudaStream_t stream);
+int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                    const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg& cfg, void* dq,
+                    void* dk, void* dv, void* ws, cudaStream_t stream);
+
+}  // namespace vardrop

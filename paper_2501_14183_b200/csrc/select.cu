@@ -1,0 +1,251 @@
+// Grouping by hash value and stratified sampling (Eq. 1, Eq. 2) in two launches, without a sort and
+// without any spin-wait.
+//
+// Launch 1 (count + finish-by-last-CTA): every CTA compares a slice of variates against a slice of keys
+// and adds, per variate n, lt[n] = #{m : key_m < key_n} and eq[n] = #{m < n : key_m = key_n} with integer
+// atomics.  lt[n] is the start of n's group in (key, index) order and eq[n] is n's rank inside its group,
+// so lt + eq is n's sorted position.  The CTA that finishes last for a hash row scatters the members,
+// scans the group heads into dense group ids / offsets, and draws each member's Philox priority.
+// Launch 2 (rank in group + finish-by-last-CTA): every member counts the members of its own group with a
+// smaller (priority, rank) pair; it is kept when that count is below the group's quota.  The last CTA of a
+// hash row compacts the kept variates into sel_idx / inv_idx with one scan.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace vardrop {
+
+namespace {
+
+constexpr int kSelThreads = 256;
+constexpr int kKeyChunk = 128;     // keys compared per CTA in launch 1
+
+struct SelectParams {
+    const uint64_t* keys;
+    int32_t *group_id, *group_offsets, *members, *n_groups, *sel_idx, *n_sel, *inv_idx;
+    // workspace
+    int* status;
+    unsigned int* done1;   // [S]
+    unsigned int* done2;   // [S]
+    int32_t* lt;           // [S, N]
+    int32_t* eq;           // [S, N]
+    uint32_t* prio;        // [S, N] priority by sorted position
+    int32_t* keep;         // [S, N] by variate
+    int S, N, gs;
+    long long rate_ppm;
+    uint32_t seed_lo, seed_hi, step;
+};
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies, xors with the key, and a
+// Weyl key schedule.  Returns word 0 of the output block.
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+__device__ __forceinline__ int quota_of(int size, int gs, long long rate_ppm) {
+    long long by_rate = (static_cast<long long>(size) * rate_ppm + 999999ll) / 1000000ll;
+    if (by_rate < 1) by_rate = 1;
+    long long q = size;
+    if (gs > 0 && gs < q) q = gs;
+    if (by_rate < q) q = by_rate;
+    return static_cast<int>(q);
+}
+
+// Inclusive scan of one int per thread across the CTA (kSelThreads threads); returns this thread's inclusive value
+// and the CTA total through `total`.
+__device__ __forceinline__ int block_scan_inclusive(int v, int* warp_sums, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += o;
+    }
+    __syncthreads();
+    if (lane == 31) warp_sums[warp] = v;
+    __syncthreads();
+    int base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kSelThreads / 32; ++w) {
+        const int s = warp_sums[w];
+        if (w < warp) base += s;
+        tot += s;
+    }
+    *total = tot;
+    return v + base;
+}
+
+// True in every thread of exactly one CTA per hash row: the one whose arrival completes the count.
+__device__ __forceinline__ bool last_cta_of_row(unsigned int* counter, unsigned int ctas_per_row, int* flag_smem) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int prev = atomicAdd(counter, 1u);
+        *flag_smem = (prev + 1u == ctas_per_row);
+    }
+    __syncthreads();
+    const bool last = *flag_smem != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectParams P) {
+    __shared__ uint64_t skeys[kKeyChunk];
+    __shared__ int warp_sums[kSelThreads / 32];
+    __shared__ int flag;
+    const int s = blockIdx.z, N = P.N;
+    const uint64_t* keys = P.keys + static_cast<size_t>(s) * N;
+    int32_t* lt = P.lt + static_cast<size_t>(s) * N;
+    int32_t* eq = P.eq + static_cast<size_t>(s) * N;
+    const int n = blockIdx.x * kSelThreads + threadIdx.x;
+    const int m0 = blockIdx.y * kKeyChunk;
+    const int mcount = min(kKeyChunk, N - m0);
+    for (int i = threadIdx.x; i < mcount; i += blockDim.x) skeys[i] = keys[m0 + i];
+    __syncthreads();
+    if (n < N) {
+        const uint64_t mine = keys[n];
+        int c_lt = 0, c_eq = 0;
+        for (int i = 0; i < mcount; ++i) {
+            const uint64_t other = skeys[i];
+            c_lt += other < mine;
+            c_eq += (other == mine) & (m0 + i < n);
+        }
+        if (c_lt) atomicAdd(lt + n, c_lt);
+        if (c_eq) atomicAdd(eq + n, c_eq);
+    }
+    if (!last_cta_of_row(P.done1 + s, gridDim.x * gridDim.y, &flag)) return;
+
+    // ---- the last CTA of this hash row: members, group heads -> ids and offsets, priorities ---------------
+    int32_t* members = P.members + static_cast<size_t>(s) * N;
+    int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
+    int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
+    uint32_t* prio = P.prio + static_cast<size_t>(s) * N;
+    for (int i = threadIdx.x; i < N; i += blockDim.x) members[__ldcg(lt + i) + __ldcg(eq + i)] = i;
+    __syncthreads();
+    // scan of head flags over sorted positions; thread t owns positions [t*per, (t+1)*per)
+    const int per = (N + kSelThreads - 1) / kSelThreads;
+    const int p_begin = min(N, static_cast<int>(threadIdx.x) * per), p_end = min(N, p_begin + per);
+    int heads = 0;
+    for (int p = p_begin; p < p_end; ++p) heads += (__ldcg(eq + members[p]) == 0);
+    int total_groups = 0;
+    int g = block_scan_inclusive(heads, warp_sums, &total_groups) - heads;   // groups before p_begin
+    for (int p = p_begin; p < p_end; ++p) {
+        const int nn = members[p];
+        if (__ldcg(eq + nn) == 0) { off[g] = p; ++g; }
+        gid[nn] = g - 1;
+    }
+    for (int i = total_groups + threadIdx.x; i <= N; i += blockDim.x) off[i] = N;
+    if (threadIdx.x == 0) P.n_groups[s] = total_groups;
+    __syncthreads();
+    for (int p = threadIdx.x; p < N; p += blockDim.x) {
+        const int nn = members[p];
+        prio[p] = philox4x32_10_word0(static_cast<uint32_t>(__ldcg(eq + nn)), static_cast<uint32_t>(gid[nn]), static_cast<uint32_t>(s),
+                                      P.step, P.seed_lo, P.seed_hi);
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const SelectParams P) {
+    __shared__ int warp_sums[kSelThreads / 32];
+    __shared__ int flag;
+    const int s = blockIdx.z, N = P.N;
+    const int32_t* members = P.members + static_cast<size_t>(s) * N;
+    const int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
+    const int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
+    const uint32_t* prio = P.prio + static_cast<size_t>(s) * N;
+    int32_t* keep = P.keep + static_cast<size_t>(s) * N;
+    const int p = blockIdx.x * kSelThreads + threadIdx.x;
+    if (p < N) {
+        const int nn = members[p];
+        const int g = gid[nn];
+        const int begin = off[g], end = off[g + 1];
+        const uint32_t mine = prio[p];
+        int smaller = 0;
+        for (int o = begin; o < end; ++o) {
+            const uint32_t other = __ldg(prio + o);
+            smaller += (other < mine) | ((other == mine) & (o < p));
+        }
+        keep[nn] = smaller < quota_of(end - begin, P.gs, P.rate_ppm);
+    }
+    if (!last_cta_of_row(P.done2 + s, gridDim.x, &flag)) return;
+
+    // ---- the last CTA of this hash row: compaction of the kept variates in ascending index order --------
+    int32_t* sel = P.sel_idx + static_cast<size_t>(s) * N;
+    int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
+    const int per = (N + kSelThreads - 1) / kSelThreads;
+    const int n_begin = min(N, static_cast<int>(threadIdx.x) * per), n_end = min(N, n_begin + per);
+    int cnt = 0;
+    for (int i = n_begin; i < n_end; ++i) cnt += __ldcg(keep + i);
+    int total = 0;
+    int pos = block_scan_inclusive(cnt, warp_sums, &total) - cnt;
+    for (int i = n_begin; i < n_end; ++i) {
+        if (__ldcg(keep + i)) { sel[pos] = i; inv[i] = pos; ++pos; } else inv[i] = -1;
+    }
+    for (int i = total + threadIdx.x; i < N; i += blockDim.x) sel[i] = -1;
+    if (threadIdx.x == 0) P.n_sel[s] = total;
+}
+
+struct SelectWs {
+    size_t done1, done2, lt, eq, prio, keep, total, zero_begin, zero_bytes;
+};
+SelectWs select_layout(int S, int N) {
+    SelectWs w;
+    size_t o = kWsHeaderBytes;
+    w.zero_begin = o;
+    w.done1 = o; o += align_up(sizeof(unsigned int) * S, 16);
+    w.done2 = o; o += align_up(sizeof(unsigned int) * S, 16);
+    w.lt = o;    o += align_up(sizeof(int32_t) * S * N, 16);
+    w.eq = o;    o += align_up(sizeof(int32_t) * S * N, 16);
+    w.zero_bytes = o - w.zero_begin;
+    w.prio = o;  o += align_up(sizeof(uint32_t) * S * N, 16);
+    w.keep = o;  o += align_up(sizeof(int32_t) * S * N, 16);
+    w.total = o;
+    return w;
+}
+
+}  // namespace
+
+int select_validate(const vardrop_select_cfg& c) {
+    if (c.S < 1 || c.S > 65535) return fail(VARDROP_ERR_INVALID_ARG, "select: S=%d outside 1..65535", c.S);
+    if (c.N < 1 || c.N > 65536) return fail(VARDROP_ERR_INVALID_ARG, "select: N=%d outside 1..65536", c.N);
+    if (!(c.rate > 0.0) || c.rate > 1.0) return fail(VARDROP_ERR_INVALID_ARG, "select: rate=%g outside (0, 1]", c.rate);
+    return VARDROP_OK;
+}
+
+size_t select_workspace_bytes(const vardrop_select_cfg& c) { return select_layout(c.S, c.N).total; }
+
+int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* group_id, int32_t* group_offsets, int32_t* members,
+                  int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, void* ws, cudaStream_t stream) {
+    const SelectWs w = select_layout(c.S, c.N);
+    char* base = static_cast<char*>(ws);
+    SelectParams P{};
+    P.keys = keys; P.group_id = group_id; P.group_offsets = group_offsets; P.members = members; P.n_groups = n_groups;
+    P.sel_idx = sel_idx; P.n_sel = n_sel; P.inv_idx = inv_idx;
+    P.status = reinterpret_cast<int*>(base);
+    P.done1 = reinterpret_cast<unsigned int*>(base + w.done1);
+    P.done2 = reinterpret_cast<unsigned int*>(base + w.done2);
+    P.lt = reinterpret_cast<int32_t*>(base + w.lt);
+    P.eq = reinterpret_cast<int32_t*>(base + w.eq);
+    P.prio = reinterpret_cast<uint32_t*>(base + w.prio);
+    P.keep = reinterpret_cast<int32_t*>(base + w.keep);
+    P.S = c.S; P.N = c.N; P.gs = c.gs;
+    P.rate_ppm = llround(c.rate * 1.0e6);
+    P.seed_lo = static_cast<uint32_t>(c.seed & 0xFFFFFFFFu);
+    P.seed_hi = static_cast<uint32_t>(c.seed >> 32);
+    P.step = c.step;
+    if (int st = check_cuda(cudaMemsetAsync(base, 0, w.zero_begin + w.zero_bytes, stream), "select: clear counters")) return st;
+    const dim3 grid1((c.N + kSelThreads - 1) / kSelThreads, (c.N + kKeyChunk - 1) / kKeyChunk, c.S);
+    select_count_kernel<<<grid1, kSelThreads, 0, stream>>>(P);
+    if (int st = check_cuda(cudaGetLastError(), "select: count launch")) return st;
+    const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
+    select_sample_kernel<<<grid2, kSelThreads, 0, stream>>>(P);
+    return check_cuda(cudaGetLastError(), "select: sample launch");
+}
+
+}  // namespace vardrop

@@ -1,0 +1,146 @@
+// C ABI of the library: argument checks, workspace carving, status text.  All arithmetic lives in the
+// kernel translation units; nothing here allocates device memory or synchronises.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace vardrop {
+
+static thread_local char g_last_error[512] = "";
+
+int fail(int status, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+int check_cuda(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return VARDROP_OK;
+    return fail(VARDROP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static int check_ptr(const void* p, const char* name, bool required) {
+    if (!p) return required ? fail(VARDROP_ERR_INVALID_ARG, "%s is NULL", name) : VARDROP_OK;
+    if (!aligned16(p)) return fail(VARDROP_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    return VARDROP_OK;
+}
+
+static int check_ws(const void* ws, size_t have, size_t need) {
+    if (int st = check_ptr(ws, "ws", true)) return st;
+    if (have < need) return fail(VARDROP_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", have, need);
+    return VARDROP_OK;
+}
+
+}  // namespace vardrop
+
+using namespace vardrop;
+
+#define VD_CHECK(expr) do { if (int st_ = (expr)) return st_; } while (0)
+
+extern "C" {
+
+const char* vardrop_status_string(int status) {
+    switch (status) {
+        case VARDROP_OK: return "ok";
+        case VARDROP_ERR_INVALID_ARG: return "invalid argument";
+        case VARDROP_ERR_UNSUPPORTED: return "unsupported shape";
+        case VARDROP_ERR_WORKSPACE: return "workspace too small";
+        case VARDROP_ERR_CUDA: return "CUDA error";
+        case VARDROP_ERR_TIMEOUT: return "bounded device wait timed out";
+        case VARDROP_ERR_NONFINITE: return "non-finite amplitude";
+        default: return "unknown status";
+    }
+}
+
+const char* vardrop_last_error(void) { return g_last_error; }
+const char* vardrop_version(void) { return "0.1"; }
+
+size_t vardrop_hash_workspace_bytes(const vardrop_hash_cfg* cfg) { return cfg ? hash_workspace_bytes(*cfg) : 0; }
+
+int vardrop_hash(const float* x, const vardrop_hash_cfg* cfg, uint64_t* keys, int32_t* freqs, float* amp_dbg, void* ws,
+                 size_t ws_bytes, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    int f_lo, f_hi;
+    VD_CHECK(hash_validate(*cfg, &f_lo, &f_hi));
+    VD_CHECK(check_ptr(x, "x", true));
+    VD_CHECK(check_ptr(keys, "keys", true));
+    VD_CHECK(check_ptr(freqs, "freqs", false));
+    VD_CHECK(check_ptr(amp_dbg, "amp_dbg", false));
+    VD_CHECK(check_ws(ws, ws_bytes, hash_workspace_bytes(*cfg)));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    VD_CHECK(check_cuda(cudaMemsetAsync(ws, 0, sizeof(int), s), "hash: clear status"));
+    return hash_launch(x, *cfg, keys, freqs, amp_dbg, static_cast<int*>(ws), s);
+}
+
+size_t vardrop_select_workspace_bytes(const vardrop_select_cfg* cfg) {
+    if (!cfg || select_validate(*cfg) != VARDROP_OK) return 0;
+    return select_workspace_bytes(*cfg);
+}
+
+int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t* group_id, int32_t* group_offsets,
+                   int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, void* ws,
+                   size_t ws_bytes, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(select_validate(*cfg));
+    VD_CHECK(check_ptr(keys, "keys", true));
+    VD_CHECK(check_ptr(group_id, "group_id", true));
+    VD_CHECK(check_ptr(group_offsets, "group_offsets", true));
+    VD_CHECK(check_ptr(members, "members", true));
+    VD_CHECK(check_ptr(n_groups, "n_groups", true));
+    VD_CHECK(check_ptr(sel_idx, "sel_idx", true));
+    VD_CHECK(check_ptr(n_sel, "n_sel", true));
+    VD_CHECK(check_ptr(inv_idx, "inv_idx", true));
+    VD_CHECK(check_ws(ws, ws_bytes, select_workspace_bytes(*cfg)));
+    return select_launch(keys, *cfg, group_id, group_offsets, members, n_groups, sel_idx, n_sel, inv_idx, ws,
+                         static_cast<cudaStream_t>(stream));
+}
+
+size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg) {
+    if (!cfg || attn_validate(*cfg) != VARDROP_OK) return 0;
+    return attn_workspace_bytes(*cfg);
+}
+
+int vardrop_attn_fwd(const void* q, const void* k, const void* v, const int32_t* sel_idx, const int32_t* n_sel,
+                     const vardrop_attn_cfg* cfg, void* o, float* lse, void* ws, size_t ws_bytes, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(attn_validate(*cfg));
+    VD_CHECK(check_ptr(q, "q", true));
+    VD_CHECK(check_ptr(k, "k", true));
+    VD_CHECK(check_ptr(v, "v", true));
+    VD_CHECK(check_ptr(sel_idx, "sel_idx", false));
+    if (sel_idx) VD_CHECK(check_ptr(n_sel, "n_sel", true));
+    VD_CHECK(check_ptr(o, "o", true));
+    VD_CHECK(check_ptr(lse, "lse", true));
+    VD_CHECK(check_ws(ws, ws_bytes, attn_workspace_bytes(*cfg)));
+    return attn_fwd_launch(q, k, v, sel_idx, n_sel, *cfg, o, lse, ws, static_cast<cudaStream_t>(stream));
+}
+
+int vardrop_attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
+                     const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg* cfg,
+                     void* dq, void* dk, void* dv, void* ws, size_t ws_bytes, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(attn_validate(*cfg));
+    VD_CHECK(check_ptr(q, "q", true));
+    VD_CHECK(check_ptr(k, "k", true));
+    VD_CHECK(check_ptr(v, "v", true));
+    VD_CHECK(check_ptr(o, "o", true));
+    VD_CHECK(check_ptr(lse, "lse", true));
+    VD_CHECK(check_ptr(d_o, "d_o", true));
+    VD_CHECK(check_ptr(sel_idx, "sel_idx", false));
+    if (sel_idx) {
+        VD_CHECK(check_ptr(n_sel, "n_sel", true));
+        VD_CHECK(check_ptr(inv_idx, "inv_idx", true));
+    }
+    VD_CHECK(check_ptr(dq, "dq", true));
+    VD_CHECK(check_ptr(dk, "dk", true));
+    VD_CHECK(check_ptr(dv, "dv", true));
+    VD_CHECK(check_ws(ws, ws_bytes, attn_workspace_bytes(*cfg)));
+    return attn_bwd_launch(q, k, v, o, lse, d_o, sel_idx, n_sel, inv_idx, *cfg, dq, dk, dv, ws, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

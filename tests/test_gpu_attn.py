@@ -1,0 +1,114 @@
+"""Parity of vardrop_attn_fwd / vardrop_attn_bwd (bf16 tensor-core kernels) with the fp64 oracle.
+Tolerance: max-abs 2e-2 and mean-abs 2e-3 on outputs and gradients."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_14183_b200 import binding as vd
+from util import assert_attn_close, bf16_tokens
+
+pytestmark = pytest.mark.gpu
+
+
+def run_attention(dev, B, N, H, D, sel, poison=True):
+    """Runs forward and backward through the C ABI.  `sel` is None (all tokens) or a sorted int array.
+    Returns o[B,Ns,H,D], lse[B,H,Ns], dq, dk, dv (numpy, float64) and the device status."""
+    q, k, v, d_full = dev
+    cfg = vd.AttnCfg(B, N, H, D, 0.0)
+    ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
+    if poison:
+        ws.view(torch.int16).fill_(0x7FC1)        # bf16 NaN pattern everywhere in the scratch
+    fill = float("nan") if poison else 0.0
+    o = torch.full((B, N, H, D), fill, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, H, N), fill, dtype=torch.float32, device="cuda")
+    if sel is None:
+        Ns, sel_t, nsel_t, inv_t = N, None, None, None
+        d_o = d_full
+    else:
+        Ns = len(sel)
+        sel_pad = np.full(N, -1, np.int32); sel_pad[:Ns] = sel
+        inv = np.full(N, -1, np.int32); inv[sel] = np.arange(Ns, dtype=np.int32)
+        sel_t = torch.from_numpy(sel_pad).cuda(); inv_t = torch.from_numpy(inv).cuda()
+        nsel_t = torch.tensor([Ns], dtype=torch.int32, device="cuda")
+        d_o = torch.full((B, N, H, D), fill, dtype=torch.bfloat16, device="cuda")      # rows past Ns may hold anything
+        d_o[:, :Ns] = d_full[:, :Ns]
+    vd.vardrop_attn_fwd(q, k, v, sel_t, nsel_t, cfg, o, lse, ws)
+    dq, dk, dv = (torch.full((B, N, H, D), fill, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, sel_t, nsel_t, inv_t, cfg, dq, dk, dv, ws)
+    torch.cuda.synchronize()
+    status = vd.ws_status(ws)
+    f = lambda t: t.double().cpu().numpy()
+    return f(o)[:, :Ns], f(lse)[:, :, :Ns], f(dq), f(dk), f(dv), status, (o, lse)
+
+
+def check_case(B, N, H, D, sel, std, seed):
+    dev, ref = bf16_tokens(B, N, H, D, std, seed)
+    o, lse, dq, dk, dv, status, raw = run_attention(dev, B, N, H, D, sel)
+    assert status == vd.OK
+    Ns = N if sel is None else len(sel)
+    wo, wl = oracle.attn_fwd(ref[0], ref[1], ref[2], sel)
+    assert_attn_close(o, wo, "o")
+    assert_attn_close(lse, wl, "lse")
+    wq, wk, wv = oracle.attn_bwd(ref[0], ref[1], ref[2], ref[3][:, :Ns], sel)
+    assert_attn_close(dq, wq, "dq")
+    assert_attn_close(dk, wk, "dk")
+    assert_attn_close(dv, wv, "dv")
+    if sel is not None:
+        dropped = np.setdiff1d(np.arange(N), sel)
+        for g in (dq, dk, dv):
+            assert np.all(g[:, dropped] == 0.0)                      # exact zeros at dropped variates
+        # rows of o / lse past n_sel are left untouched (still the NaN fill)
+        assert torch.isnan(raw[0][:, Ns:].float()).all() and torch.isnan(raw[1][:, :, Ns:]).all()
+
+
+def pick(N, Ns, seed):
+    return np.sort(np.random.default_rng(seed).choice(N, size=Ns, replace=False)).astype(np.int32)
+
+
+@pytest.mark.parametrize("B,N,H,D,Ns", [
+    (2, 21, 4, 32, 11), (1, 7, 1, 64, 1), (2, 40, 2, 64, 40), (2, 300, 2, 64, 128), (1, 300, 3, 64, 129),
+    (2, 321, 2, 64, 97), (1, 600, 2, 64, 300), (1, 500, 2, 32, 257), (3, 130, 1, 64, 127)])
+@pytest.mark.parametrize("std", [1.0, 0.3536])
+def test_attention_selected(B, N, H, D, Ns, std):
+    check_case(B, N, H, D, pick(N, Ns, seed=N + Ns), std, seed=N * 7 + Ns)
+
+
+@pytest.mark.parametrize("B,N,H,D", [(2, 21, 4, 32), (1, 128, 2, 64), (2, 200, 2, 64), (1, 385, 2, 64), (1, 256, 1, 32), (1, 1, 1, 64)])
+def test_attention_all_tokens(B, N, H, D):
+    check_case(B, N, H, D, None, 1.0, seed=N)
+
+
+def test_attention_identity_selection_equals_all_token_path():
+    B, N, H, D = 1, 200, 2, 64
+    dev, _ = bf16_tokens(B, N, H, D, 1.0, seed=3)
+    a = run_attention(dev, B, N, H, D, None, poison=False)
+    b = run_attention(dev, B, N, H, D, np.arange(N, dtype=np.int32), poison=False)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])       # forward is bit-reproducible
+    for x, y in zip(a[3:5], b[3:5]):
+        assert np.array_equal(x, y)                                        # dk, dv too
+    np.testing.assert_allclose(a[2], b[2], atol=1e-2)                      # dq: atomics, order may differ
+
+
+def test_attention_forward_is_deterministic():
+    B, N, H, D = 2, 300, 2, 64
+    dev, _ = bf16_tokens(B, N, H, D, 1.0, seed=4)
+    sel = pick(N, 200, 1)
+    a = run_attention(dev, B, N, H, D, sel, poison=False)
+    b = run_attention(dev, B, N, H, D, sel, poison=False)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[3], b[3]) and np.array_equal(a[4], b[4])
+
+
+def test_attention_argument_errors():
+    q = torch.zeros((1, 8, 1, 64), dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((1, 1, 8), device="cuda")
+    ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(vd.AttnCfg(1, 8, 1, 64, 0.0)))
+    with pytest.raises(vd.VardropError) as e:
+        vd.vardrop_attn_fwd(q, q, q, None, None, vd.AttnCfg(1, 8, 1, 128, 0.0), q, lse, ws)
+    assert e.value.status == vd.ERR_UNSUPPORTED
+    with pytest.raises(vd.VardropError) as e:
+        vd.vardrop_attn_fwd(q, q, q, None, None, vd.AttnCfg(1, 8, 1, 64, 0.0), q, lse, ws[:256])
+    assert e.value.status == vd.ERR_WORKSPACE
+    with pytest.raises(vd.VardropError) as e:
+        vd.vardrop_attn_fwd(q, None, q, None, None, vd.AttnCfg(1, 8, 1, 64, 0.0), q, lse, ws)
+    assert e.value.status == vd.ERR_INVALID_ARG

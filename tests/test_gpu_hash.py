@@ -1,0 +1,132 @@
+"""Parity of vardrop_hash (CUDA, fp32 FFT) with the fp64 oracle: keys and ranked bins bit-exact on rank-gap filtered
+inputs, flip counts reported on unfiltered ones, mean amplitudes within fp32 rounding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_14183_b200 import binding as vd
+from paper_2501_14183_b200 import inputs
+from util import RANK_GAP, gap_filtered_windows
+
+pytestmark = pytest.mark.gpu
+
+
+def run_hash(x, k, f_lo=0, f_hi=0, scope=0, want_amp=True):
+    B, N, L = x.shape
+    cfg = vd.HashCfg(B, N, L, k, f_lo, f_hi, scope)
+    xd = torch.from_numpy(x).cuda()
+    keys, freqs, amp = vd.alloc_hash_outputs(cfg, want_amp=want_amp)
+    ws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(cfg))
+    vd.vardrop_hash(xd, cfg, keys, freqs, amp, ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.OK
+    return keys.cpu().numpy().view(np.uint64), freqs.cpu().numpy(), None if amp is None else amp.cpu().numpy()
+
+
+def random_periodic(B, N, L, k, seed):
+    """sums of k+2 sinusoids at random (non-integer) periods with a geometric amplitude ladder + noise."""
+    rng = np.random.default_rng(seed)
+    t = np.arange(L)
+    x = np.zeros((B, N, L))
+    nb = L // 2 + 1
+    hi = max(3, (nb + 1) // 2)
+    for i in range(k + 2):
+        f = rng.uniform(1, hi - 1, size=(1, N, 1))
+        a = (0.55 ** i) * rng.uniform(0.8, 1.2, size=(1, N, 1))
+        ph = rng.uniform(0, 2 * np.pi, size=(B, N, 1))
+        x += a * np.sin(2 * np.pi * f * t / L + ph)
+    x += rng.normal(0, 0.05, size=x.shape)
+    return x.astype(np.float32)
+
+
+SHAPES = [
+    # B, N, L, k, scope
+    (4, 21, 96, 2, 0), (1, 1, 96, 3, 0), (3, 37, 96, 3, 0), (32, 50, 96, 3, 0), (5, 33, 336, 4, 0), (16, 9, 720, 5, 0),
+    (7, 19, 720, 5, 0), (2, 13, 48, 2, 0), (3, 11, 30, 2, 0), (2, 5, 14, 1, 0), (4, 8, 64, 3, 0), (3, 6, 2048, 5, 0),
+    (70, 3, 96, 3, 0), (4, 21, 96, 2, 1), (3, 10, 336, 4, 1), (5, 7, 720, 5, 1), (1, 300, 96, 3, 0), (2, 4, 210, 3, 0),
+]
+
+
+@pytest.mark.parametrize("B,N,L,k,scope", SHAPES)
+def test_hash_parity_small(B, N, L, k, scope):
+    nb = L // 2 + 1
+    if (nb + 1) // 2 - 1 < k + 1:
+        f_lo, f_hi = 0, nb
+    else:
+        f_lo, f_hi = 0, 0
+    x = random_periodic(B, N, L, k, seed=B * 1000 + N * 10 + L)
+    x, keys, freqs, abar, _ = gap_filtered_windows(x, k, f_lo, f_hi, scope)
+    gk, gf, ga = run_hash(x, k, f_lo, f_hi, scope)
+    assert np.array_equal(gf, freqs)
+    assert np.array_equal(gk, keys)
+    np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
+
+
+@pytest.mark.parametrize("name", ["tiny", "elec", "traffic", "long", "scale"])
+def test_hash_parity_workloads(name):
+    w = inputs.WORKLOADS[name]
+    x0 = inputs.make_windows(w)
+    # unfiltered: report how many hashes flip against fp64 (none expected outside the gap band)
+    keys0, _, abar0 = oracle.hash(x0, w.k)
+    gk0, _, _ = run_hash(x0, w.k, want_amp=False)
+    flips = np.nonzero(gk0[0] != keys0[0])[0]
+    gaps = oracle.rank_gaps(abar0, w.k)[0]
+    print(f"[{name}] unfiltered tie flips: {len(flips)} of {w.N}; variates inside the gap band: {(gaps <= RANK_GAP).sum()}")
+    assert np.all(gaps[flips] <= RANK_GAP)          # a flip is only allowed where the ranking is a near-tie
+    # filtered: bit-exact
+    x, keys, freqs, abar, n_rep = gap_filtered_windows(x0, w.k)
+    gk, gf, ga = run_hash(x, w.k)
+    assert np.array_equal(gk, keys) and np.array_equal(gf, freqs)
+    np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
+
+
+def test_hash_band_options_and_debug_outputs_optional():
+    x = random_periodic(4, 16, 96, 3, seed=5)
+    for f_lo, f_hi in [(0, 49), (1, 25), (0, 25), (1, 26), (5, 20)]:
+        xf, keys, freqs, abar, _ = gap_filtered_windows(x, 3, f_lo, f_hi)
+        gk, gf, ga = run_hash(xf, 3, f_lo, f_hi)
+        assert np.array_equal(gk, keys) and np.array_equal(gf, freqs)
+    # freqs / amp_dbg may be NULL
+    cfg = vd.HashCfg(4, 16, 96, 3, 0, 0, 0)
+    keys_t, _, _ = vd.alloc_hash_outputs(cfg, want_freqs=False)
+    ws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(cfg))
+    xf, keys, _, _, _ = gap_filtered_windows(x, 3)
+    vd.vardrop_hash(torch.from_numpy(xf).cuda(), cfg, keys_t, None, None, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(keys_t.cpu().numpy().view(np.uint64), keys)
+
+
+def test_hash_is_deterministic():
+    w = inputs.WORKLOADS["elec"]
+    x = inputs.make_windows(w)
+    a = run_hash(x, w.k)
+    b = run_hash(x, w.k)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[2], b[2])
+
+
+def test_hash_nonfinite_input_sets_status():
+    x = random_periodic(2, 4, 96, 3, seed=1)
+    x[1, 2, 17] = np.nan
+    cfg = vd.HashCfg(2, 4, 96, 3, 0, 0, 0)
+    keys, freqs, amp = vd.alloc_hash_outputs(cfg)
+    ws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(cfg))
+    vd.vardrop_hash(torch.from_numpy(x).cuda(), cfg, keys, freqs, amp, ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.ERR_NONFINITE
+
+
+def test_hash_argument_errors():
+    x = torch.zeros((2, 4, 96), device="cuda")
+    ws = vd.alloc_ws(256)
+    keys = torch.empty((1, 4), dtype=torch.int64, device="cuda")
+    for cfg, status in [(vd.HashCfg(2, 4, 96, 0, 0, 0, 0), vd.ERR_INVALID_ARG), (vd.HashCfg(2, 4, 96, 6, 0, 0, 0), vd.ERR_INVALID_ARG),
+                        (vd.HashCfg(2, 4, 94, 3, 0, 0, 0), vd.ERR_UNSUPPORTED),      # 94 = 2 * 47
+                        (vd.HashCfg(2, 4, 96, 3, 10, 12, 0), vd.ERR_INVALID_ARG), (vd.HashCfg(2, 4, 96, 3, 0, 60, 0), vd.ERR_INVALID_ARG),
+                        (vd.HashCfg(2, 4, 96, 3, 0, 0, 2), vd.ERR_INVALID_ARG)]:
+        with pytest.raises(vd.VardropError) as e:
+            vd.vardrop_hash(x, cfg, keys, None, None, ws)
+        assert e.value.status == status
+    with pytest.raises(vd.VardropError) as e:
+        vd.vardrop_hash(None, vd.HashCfg(2, 4, 96, 3, 0, 0, 0), keys, None, None, ws)
+    assert e.value.status == vd.ERR_INVALID_ARG

@@ -1,0 +1,92 @@
+"""Parity of vardrop_select with the oracle: every output bit-exact (integer work)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_14183_b200 import binding as vd
+from paper_2501_14183_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def run_select(keys, gs, rate, seed, step):
+    keys = np.atleast_2d(keys)
+    S, N = keys.shape
+    cfg = vd.SelectCfg(S, N, gs, rate, seed, step)
+    kd = torch.from_numpy(keys.view(np.int64)).cuda()
+    out = vd.alloc_select_outputs(cfg)
+    ws = vd.alloc_ws(vd.vardrop_select_workspace_bytes(cfg))
+    vd.vardrop_select(kd, cfg, out["group_id"], out["group_offsets"], out["members"], out["n_groups"], out["sel_idx"],
+                      out["n_sel"], out["inv_idx"], ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.OK
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def check(keys, gs, rate, seed, step):
+    want = oracle.select(keys, gs, rate, seed, step)
+    got = run_select(keys, gs, rate, seed, step)
+    for name in ("n_groups", "n_sel", "group_id", "group_offsets", "members", "sel_idx", "inv_idx"):
+        assert np.array_equal(got[name], want[name]), name
+    return got
+
+
+@pytest.mark.parametrize("N,G", [(1, 1), (2, 2), (21, 4), (127, 9), (128, 128), (129, 1), (257, 30), (321, 40), (862, 60),
+                                 (1000, 1000), (3000, 7), (8192, 512)])
+@pytest.mark.parametrize("gs,rate", [(10, 1.0), (0, 0.2), (3, 0.5)])
+def test_select_parity(N, G, gs, rate):
+    keys = inputs.make_keys(N, G, k=4, f_hi=85, seed=N + G)
+    check(keys, gs, rate, seed=0xC0FFEE1234567, step=N % 7)
+
+
+def test_select_degenerate_groups():
+    same = np.full(2000, (5 << 24) | (9 << 12) | 2, dtype=np.uint64)
+    got = check(same, 10, 1.0, seed=1, step=0)
+    assert got["n_groups"][0] == 1 and got["n_sel"][0] == 10
+    distinct = np.arange(1, 1501, dtype=np.uint64)[np.random.default_rng(0).permutation(1500)]
+    got = check(distinct, 10, 1.0, seed=1, step=0)
+    assert got["n_groups"][0] == 1500 and got["n_sel"][0] == 1500
+    check(np.full(300, 0xFFFFFFFFFFFFFFF, dtype=np.uint64), 0, 0.1, seed=3, step=9)     # 60-bit keys (k = 5)
+
+
+def test_select_multiple_scopes():
+    rows = np.stack([inputs.make_keys(500, 20 + s, k=3, f_hi=25, seed=s) for s in range(5)])
+    got = check(rows, 5, 1.0, seed=77, step=3)
+    assert len(set(got["n_sel"].tolist())) > 1
+
+
+def test_select_paper_hyperparameters():
+    # (k, gs) of Appendix E on keys hashed from the synthetic workloads
+    for name, gs in (("elec", 10), ("traffic", 10), ("tiny", 5)):
+        w = inputs.WORKLOADS[name]
+        keys, _, _ = oracle.hash(inputs.make_windows(w, B=4), w.k)
+        got = check(keys, gs, 1.0, seed=20250114, step=1)
+        sizes = np.diff(got["group_offsets"][0][: got["n_groups"][0] + 1])
+        assert got["n_sel"][0] == np.minimum(sizes, gs).sum()           # Eq. 1 summed over groups
+
+
+def test_select_reproducible_and_step_dependent():
+    keys = inputs.make_keys(862, 60, k=3, f_hi=25, seed=2)
+    a = run_select(keys, 0, 0.2, seed=5, step=10)
+    b = run_select(keys, 0, 0.2, seed=5, step=10)
+    c = run_select(keys, 0, 0.2, seed=5, step=11)
+    assert np.array_equal(a["sel_idx"], b["sel_idx"])
+    assert not np.array_equal(a["sel_idx"], c["sel_idx"])
+    assert a["n_sel"][0] == c["n_sel"][0]
+
+
+def test_select_argument_errors():
+    keys = torch.zeros((1, 8), dtype=torch.int64, device="cuda")
+    cfg = vd.SelectCfg(1, 8, 0, 0.5, 1, 0)
+    out = vd.alloc_select_outputs(cfg)
+    args = (out["group_id"], out["group_offsets"], out["members"], out["n_groups"], out["sel_idx"], out["n_sel"], out["inv_idx"])
+    small = vd.alloc_ws(256)
+    with pytest.raises(vd.VardropError) as e:
+        vd.vardrop_select(keys, cfg, *args, small[:128])
+    assert e.value.status == vd.ERR_WORKSPACE
+    ws = vd.alloc_ws(vd.vardrop_select_workspace_bytes(cfg))
+    for bad in (vd.SelectCfg(1, 8, 0, 0.0, 1, 0), vd.SelectCfg(1, 8, 0, 1.5, 1, 0), vd.SelectCfg(1, 0, 0, 0.5, 1, 0), vd.SelectCfg(0, 8, 0, 0.5, 1, 0)):
+        with pytest.raises(vd.VardropError) as e:
+            vd.vardrop_select(keys, bad, *args, ws)
+        assert e.value.status == vd.ERR_INVALID_ARG
