@@ -51,6 +51,24 @@ const char* vardrop_last_error(void);
 const char* vardrop_version(void);
 
 /* ------------------------------------------------------------------------------------------------
+ * Measurement aids (no counterpart in the paper).
+ *   vardrop_launch_count          kernels this library has launched in this process so far.
+ *   vardrop_profile_enable(on)    arms (1) or disarms (0) the per-kernel timer and drops what it had collected.
+ *                                 While armed every kernel launch is bracketed by a pair of CUDA events on its
+ *                                 stream (host-side objects owned by the library), which costs a little idle
+ *                                 time between kernels: arm it only for profiling passes.
+ *   vardrop_profile_kernels       number of distinct kernels; ids are 0 .. count-1.
+ *   vardrop_profile_kernel_name   name of kernel `id`.
+ *   vardrop_profile_read          waits for the recorded events of kernel `id` and returns the sum of their
+ *                                 durations (host pointers: total_ms, launches).
+ * ---------------------------------------------------------------------------------------------- */
+long long vardrop_launch_count(void);
+int vardrop_profile_enable(int on);
+int vardrop_profile_kernels(void);
+const char* vardrop_profile_kernel_name(int id);
+int vardrop_profile_read(int id, double* total_ms, long long* launches);
+
+/* ------------------------------------------------------------------------------------------------
  * k-dominant frequency hashing -- Algorithm 1 ("k-Dominant Frequency Hashing") and Definition 1.
  *
  *   step 1  amplitude spectrum A[b,n,f] = |sum_t x[b,n,t] exp(-2 pi i f t / L)| of every window

@@ -42,7 +42,8 @@ class VardropError(RuntimeError):
 
 EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_hash_workspace_bytes", "vardrop_hash",
            "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
-           "vardrop_attn_bwd")
+           "vardrop_attn_bwd", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
+           "vardrop_profile_kernel_name", "vardrop_profile_read")
 
 
 def load() -> C.CDLL:
@@ -66,6 +67,11 @@ def load() -> C.CDLL:
         lib.vardrop_attn_fwd.argtypes = [C.c_void_p] * 9 + [C.c_size_t, C.c_void_p]
         lib.vardrop_attn_bwd.restype = C.c_int
         lib.vardrop_attn_bwd.argtypes = [C.c_void_p] * 14 + [C.c_size_t, C.c_void_p]
+        lib.vardrop_launch_count.restype = C.c_longlong
+        lib.vardrop_profile_kernel_name.restype = C.c_char_p
+        lib.vardrop_profile_kernel_name.argtypes = [C.c_int]
+        lib.vardrop_profile_enable.argtypes = [C.c_int]
+        lib.vardrop_profile_read.argtypes = [C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
         _lib = lib
     return _lib
 
@@ -115,6 +121,25 @@ def vardrop_attn_bwd(q, k, v, o, lse, d_o, sel_idx, n_sel, inv_idx, cfg: AttnCfg
     _check(load().vardrop_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(sel_idx), _ptr(n_sel),
                                    _ptr(inv_idx), C.byref(cfg), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws),
                                    ws.numel() * ws.element_size(), _stream()), "vardrop_attn_bwd")
+
+
+def vardrop_launch_count() -> int:
+    return int(load().vardrop_launch_count())
+
+
+def vardrop_profile_enable(on: bool) -> None:
+    _check(load().vardrop_profile_enable(1 if on else 0), "vardrop_profile_enable")
+
+
+def vardrop_profile_read() -> dict:
+    """{kernel name: (total milliseconds, launches)} for everything recorded since the timer was armed."""
+    lib = load()
+    out = {}
+    for kid in range(lib.vardrop_profile_kernels()):
+        ms, n = C.c_double(0.0), C.c_longlong(0)
+        _check(lib.vardrop_profile_read(kid, C.byref(ms), C.byref(n)), "vardrop_profile_read")
+        out[lib.vardrop_profile_kernel_name(kid).decode()] = (ms.value, int(n.value))
+    return out
 
 
 def ws_status(ws) -> int:

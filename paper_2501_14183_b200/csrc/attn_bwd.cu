@@ -346,7 +346,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         const long long work = static_cast<long long>(w.Ncap) * c.H * 8;
         int gx = static_cast<int>((work + 255) / 256);
         if (gx > 1184) gx = 1184;
-        bwd_prep_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(R);
+        { LaunchScope ls_(K_BWD_PREP, stream); bwd_prep_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(R); }
         if (int st = check_cuda(cudaGetLastError(), "attention: backward prep launch")) return st;
     }
 
@@ -376,7 +376,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         if (int st = check_cuda(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
-    attn_bwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P);
+    { LaunchScope ls_(K_ATTN_BWD, stream); attn_bwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P); }
     if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
 
     FinishParams F{};
@@ -388,7 +388,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         const long long work = static_cast<long long>(c.N) * c.H * (c.D / 8);
         int gx = static_cast<int>((work + 255) / 256);
         if (gx > 1184) gx = 1184;
-        bwd_finish_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F);
+        { LaunchScope ls_(K_BWD_FINISH, stream); bwd_finish_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F); }
     }
     return check_cuda(cudaGetLastError(), "attention: backward finish launch");
 }

@@ -306,7 +306,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
         int gx = static_cast<int>((work + 255) / 256);
         if (gx > 1184) gx = 1184;
-        gather_kernel<<<dim3(gx, c.B, 3), 256, 0, stream>>>(G);
+        { LaunchScope ls_(K_GATHER, stream); gather_kernel<<<dim3(gx, c.B, 3), 256, 0, stream>>>(G); }
         if (int st = check_cuda(cudaGetLastError(), "attention: gather launch")) return st;
         if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
@@ -329,7 +329,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         if (int st = check_cuda(cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
-    attn_fwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P);
+    { LaunchScope ls_(K_ATTN_FWD, stream); attn_fwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P); }
     return check_cuda(cudaGetLastError(), "attention: forward launch");
 }
 

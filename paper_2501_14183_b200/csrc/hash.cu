@@ -351,7 +351,7 @@ int hash_launch(const float* x, const vardrop_hash_cfg& c, uint64_t* keys, int32
         attr_done_dev = dev;
     }
     const int grid = (P.rows_total + P.rows_per_cta - 1) / P.rows_per_cta;
-    hash_kernel<<<grid, kHashThreads, smem, stream>>>(P);
+    { LaunchScope ls_(K_HASH, stream); hash_kernel<<<grid, kHashThreads, smem, stream>>>(P); }
     return check_cuda(cudaGetLastError(), "hash: launch");
 }
 

@@ -9,6 +9,19 @@
 
 namespace vardrop {
 
+// Kernel identities for the launch counter and the optional per-kernel event timer (vardrop_profile_*).
+enum KernelId {
+    K_HASH = 0, K_SELECT_COUNT, K_SELECT_SAMPLE, K_GATHER, K_ATTN_FWD, K_BWD_PREP, K_ATTN_BWD, K_BWD_FINISH, K_COUNT
+};
+// Wrap a kernel launch: counts it and, when the timer is armed, brackets it with a pair of CUDA events on `stream`.
+struct LaunchScope {
+    LaunchScope(int id, cudaStream_t stream);
+    ~LaunchScope();
+    int id_;
+    cudaStream_t stream_;
+    void* stop_;
+};
+
 // hash.cu
 size_t hash_workspace_bytes(const vardrop_hash_cfg& cfg);
 int hash_validate(const vardrop_hash_cfg& cfg, int* f_lo, int* f_hi);

@@ -241,10 +241,10 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
     P.step = c.step;
     if (int st = check_cuda(cudaMemsetAsync(base, 0, w.zero_begin + w.zero_bytes, stream), "select: clear counters")) return st;
     const dim3 grid1((c.N + kSelThreads - 1) / kSelThreads, (c.N + kKeyChunk - 1) / kKeyChunk, c.S);
-    select_count_kernel<<<grid1, kSelThreads, 0, stream>>>(P);
+    { LaunchScope ls_(K_SELECT_COUNT, stream); select_count_kernel<<<grid1, kSelThreads, 0, stream>>>(P); }
     if (int st = check_cuda(cudaGetLastError(), "select: count launch")) return st;
     const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
-    select_sample_kernel<<<grid2, kSelThreads, 0, stream>>>(P);
+    { LaunchScope ls_(K_SELECT_SAMPLE, stream); select_sample_kernel<<<grid2, kSelThreads, 0, stream>>>(P); }
     return check_cuda(cudaGetLastError(), "select: sample launch");
 }
 

@@ -3,6 +3,9 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <utility>
+#include <vector>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -36,6 +39,37 @@ static int check_ws(const void* ws, size_t have, size_t need) {
     return VARDROP_OK;
 }
 
+// ---- launch counter and optional per-kernel event timer ---------------------------------------------------
+namespace {
+std::mutex g_prof_mutex;
+bool g_prof_on = false;
+long long g_launches = 0;
+std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_events[K_COUNT];   // pairs recorded since the timer was armed
+std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_free;              // pairs ready for reuse
+const char* const g_kernel_names[K_COUNT] = {"hash_kernel", "select_count_kernel", "select_sample_kernel", "gather_kernel",
+                                             "attn_fwd_kernel", "bwd_prep_kernel", "attn_bwd_kernel", "bwd_finish_kernel"};
+}  // namespace
+
+LaunchScope::LaunchScope(int id, cudaStream_t stream) : id_(id), stream_(stream), stop_(nullptr) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    ++g_launches;
+    if (!g_prof_on) return;
+    std::pair<cudaEvent_t, cudaEvent_t> ev;
+    if (!g_prof_free.empty()) {
+        ev = g_prof_free.back();
+        g_prof_free.pop_back();
+    } else if (cudaEventCreate(&ev.first) != cudaSuccess || cudaEventCreate(&ev.second) != cudaSuccess) {
+        return;
+    }
+    cudaEventRecord(ev.first, stream);
+    g_prof_events[id].push_back(ev);
+    stop_ = ev.second;
+}
+
+LaunchScope::~LaunchScope() {
+    if (stop_) cudaEventRecord(static_cast<cudaEvent_t>(stop_), stream_);
+}
+
 }  // namespace vardrop
 
 using namespace vardrop;
@@ -59,6 +93,40 @@ const char* vardrop_status_string(int status) {
 
 const char* vardrop_last_error(void) { return g_last_error; }
 const char* vardrop_version(void) { return "0.1"; }
+
+long long vardrop_launch_count(void) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    return g_launches;
+}
+
+int vardrop_profile_kernels(void) { return K_COUNT; }
+
+const char* vardrop_profile_kernel_name(int id) { return id >= 0 && id < K_COUNT ? g_kernel_names[id] : ""; }
+
+int vardrop_profile_enable(int on) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    for (int id = 0; id < K_COUNT; ++id) {
+        for (auto& ev : g_prof_events[id]) g_prof_free.push_back(ev);
+        g_prof_events[id].clear();
+    }
+    g_prof_on = on != 0;
+    return VARDROP_OK;
+}
+
+int vardrop_profile_read(int id, double* total_ms, long long* launches) {
+    if (id < 0 || id >= K_COUNT || !total_ms || !launches) return fail(VARDROP_ERR_INVALID_ARG, "profile_read: bad argument");
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    double sum = 0.0;
+    for (auto& ev : g_prof_events[id]) {
+        if (int st = check_cuda(cudaEventSynchronize(ev.second), "profile_read: event synchronize")) return st;
+        float ms = 0.f;
+        if (int st = check_cuda(cudaEventElapsedTime(&ms, ev.first, ev.second), "profile_read: elapsed time")) return st;
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = static_cast<long long>(g_prof_events[id].size());
+    return VARDROP_OK;
+}
 
 size_t vardrop_hash_workspace_bytes(const vardrop_hash_cfg* cfg) { return cfg ? hash_workspace_bytes(*cfg) : 0; }
 

@@ -1,0 +1,89 @@
+"""The whole hot path through the C ABI on the benchmark's configurations and launch shapes, against the oracle:
+hash -> select bit-exact on rank-gap filtered inputs, attention forward/backward within tolerance on sampled
+(instance, head) problems the oracle can afford."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_14183_b200 import binding as vd
+from paper_2501_14183_b200 import inputs
+from util import assert_attn_close, gap_filtered_windows
+
+pytestmark = pytest.mark.gpu
+SEED, STEP = 20250114, 5
+
+
+def run_path(w, x, toks, vardrop=True):
+    dev = [torch.from_numpy(t).cuda().to(torch.bfloat16) for t in toks]
+    q, k, v, d_o = dev
+    acfg = vd.AttnCfg(w.B, w.N, w.H, w.D, 0.0)
+    aws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(acfg))
+    o = torch.zeros_like(q)
+    lse = torch.zeros((w.B, w.H, w.N), dtype=torch.float32, device="cuda")
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    sel = None
+    if vardrop:
+        hcfg = vd.HashCfg(w.B, w.N, w.L, w.k, 0, 0, 0)
+        keys, freqs, _ = vd.alloc_hash_outputs(hcfg)
+        hws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(hcfg))
+        vd.vardrop_hash(torch.from_numpy(x).cuda(), hcfg, keys, freqs, None, hws)
+        scfg = vd.SelectCfg(1, w.N, 0, w.rate, SEED, STEP)
+        sel = vd.alloc_select_outputs(scfg)
+        sws = vd.alloc_ws(vd.vardrop_select_workspace_bytes(scfg))
+        vd.vardrop_select(keys, scfg, sel["group_id"], sel["group_offsets"], sel["members"], sel["n_groups"], sel["sel_idx"],
+                          sel["n_sel"], sel["inv_idx"], sws)
+        vd.vardrop_attn_fwd(q, k, v, sel["sel_idx"], sel["n_sel"], acfg, o, lse, aws)
+        vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, sel["sel_idx"], sel["n_sel"], sel["inv_idx"], acfg, dq, dk, dv, aws)
+        torch.cuda.synchronize()
+        assert vd.ws_status(hws) == vd.OK and vd.ws_status(sws) == vd.OK
+        sel = {k_: v_.cpu().numpy() for k_, v_ in sel.items()}
+        sel["keys"] = keys.cpu().numpy().view(np.uint64)
+    else:
+        vd.vardrop_attn_fwd(q, k, v, None, None, acfg, o, lse, aws)
+        vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, None, None, None, acfg, dq, dk, dv, aws)
+        torch.cuda.synchronize()
+    assert vd.ws_status(aws) == vd.OK
+    return dev, sel, o, lse, dq, dk, dv
+
+
+def check_attention_samples(w, dev, idx, o, lse, dq, dk, dv, pairs):
+    """Oracle on single (b, h) problems cut out of the batch."""
+    Ns = w.N if idx is None else len(idx)
+    for b, h in pairs:
+        cut = [t[b:b + 1, :, h:h + 1].double().cpu().numpy() for t in dev]
+        wo, wl = oracle.attn_fwd(cut[0], cut[1], cut[2], idx)
+        assert_attn_close(o[b:b + 1, :Ns, h:h + 1].double().cpu().numpy(), wo, f"o[{b},{h}]")
+        assert_attn_close(lse[b:b + 1, h:h + 1, :Ns].double().cpu().numpy(), wl, f"lse[{b},{h}]")
+        wq, wk, wv = oracle.attn_bwd(cut[0], cut[1], cut[2], cut[3][:, :Ns], idx)
+        assert_attn_close(dq[b:b + 1, :, h:h + 1].double().cpu().numpy(), wq, f"dq[{b},{h}]")
+        assert_attn_close(dk[b:b + 1, :, h:h + 1].double().cpu().numpy(), wk, f"dk[{b},{h}]")
+        assert_attn_close(dv[b:b + 1, :, h:h + 1].double().cpu().numpy(), wv, f"dv[{b},{h}]")
+
+
+@pytest.mark.parametrize("name", ["tiny", "elec", "traffic", "long", "scale"])
+def test_whole_path_on_workload(name):
+    w = inputs.WORKLOADS[name]
+    x, okeys, _, _, _ = gap_filtered_windows(inputs.make_windows(w), w.k)
+    toks = inputs.make_tokens(w.B, w.N, w.H, w.D, w.qkv_std, seed=w.seed + 1)
+    dev, sel, o, lse, dq, dk, dv = run_path(w, x, toks)
+    assert np.array_equal(sel["keys"], okeys)
+    want = oracle.select(okeys, 0, w.rate, SEED, STEP)
+    for key in ("n_groups", "n_sel", "group_id", "group_offsets", "members", "sel_idx", "inv_idx"):
+        assert np.array_equal(sel[key], want[key]), key
+    n_sel = int(want["n_sel"][0])
+    idx = want["sel_idx"][0, :n_sel]
+    print(f"[{name}] groups={int(want['n_groups'][0])} kept={n_sel} of {w.N} (delta={1 - n_sel / w.N:.3f})")
+    pairs = [(0, 0), (w.B - 1, w.H - 1), (w.B // 2, w.H // 2)] if name != "tiny" else [(b, h) for b in range(w.B) for h in range(w.H)]
+    check_attention_samples(w, dev, idx, o, lse, dq, dk, dv, pairs)
+    dropped = np.setdiff1d(np.arange(w.N), idx)
+    for g in (dq, dk, dv):
+        assert not g[:, torch.from_numpy(dropped).cuda()].any()               # exact zeros at every dropped variate
+
+
+@pytest.mark.parametrize("name,pairs", [("traffic", [(0, 0), (31, 7)]), ("scale", [(3, 5)])])
+def test_vardrop_off_full_attention(name, pairs):
+    w = inputs.WORKLOADS[name]
+    toks = inputs.make_tokens(w.B, w.N, w.H, w.D, w.qkv_std, seed=w.seed + 1)
+    dev, _, o, lse, dq, dk, dv = run_path(w, None, toks, vardrop=False)
+    check_attention_samples(w, dev, None, o, lse, dq, dk, dv, pairs)
