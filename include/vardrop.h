@@ -137,6 +137,30 @@ int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t*
                    void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * vardrop_select without a workspace (the paper has no counterpart; this is a packaging variant).
+ *
+ * For callers that cannot obtain device memory at the point where they select tokens: code running
+ * inside a framework whose allocator is locked or already exhausted, plug-ins that are handed
+ * input/output buffers and nothing else, or hosts that forbid cudaMalloc after start-up.  The
+ * scratch that vardrop_select takes as `ws` lives here in a fixed 400 KiB array that is part of
+ * the library image; every GPU that loads the library carries that array until the process ends.
+ *
+ * Same arguments, outputs and results as vardrop_select, minus ws / ws_bytes.
+ * Limit: S * N <= 16384; larger problems return VARDROP_ERR_UNSUPPORTED (use vardrop_select).
+ * It never calls cudaMalloc, cudaFree or any allocating routine; it issues one cudaMemsetAsync and
+ * two kernel launches on `stream`.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and caches it; make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps whatever the previous call left: the parts
+ * that must start at zero are cleared at the head of every call, so back-to-back calls on one stream
+ * are fine, but two calls whose GPU work overlaps (different streams, different threads) race and
+ * give wrong results.  There is no device status word to read back for this variant.
+ * ---------------------------------------------------------------------------------------------- */
+int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t* group_id, int32_t* group_offsets,
+                          int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx,
+                          void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Attention over the kept tokens -- Sec. 3.3 (token reduction: only the selected variate tokens enter
  * self-attention) and Eq. 3, per batch instance b and head h:
  *   Q' = q[b, sel_idx[0..n_sel), h, :] (same for K', V');  O' = softmax(Q' K'^T * sm_scale) V';

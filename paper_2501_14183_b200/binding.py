@@ -41,7 +41,7 @@ class VardropError(RuntimeError):
 
 
 EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_hash_workspace_bytes", "vardrop_hash",
-           "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
+           "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_select_static", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
            "vardrop_attn_bwd", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
            "vardrop_profile_kernel_name", "vardrop_profile_read")
 
@@ -63,6 +63,8 @@ def load() -> C.CDLL:
         lib.vardrop_hash.argtypes = [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
         lib.vardrop_select.restype = C.c_int
         lib.vardrop_select.argtypes = [C.c_void_p] * 10 + [C.c_size_t, C.c_void_p]
+        lib.vardrop_select_static.restype = C.c_int
+        lib.vardrop_select_static.argtypes = [C.c_void_p] * 10
         lib.vardrop_attn_fwd.restype = C.c_int
         lib.vardrop_attn_fwd.argtypes = [C.c_void_p] * 9 + [C.c_size_t, C.c_void_p]
         lib.vardrop_attn_bwd.restype = C.c_int
@@ -110,6 +112,14 @@ def vardrop_select(keys, cfg: SelectCfg, group_id, group_offsets, members, n_gro
     _check(load().vardrop_select(_ptr(keys), C.byref(cfg), _ptr(group_id), _ptr(group_offsets), _ptr(members), _ptr(n_groups),
                                  _ptr(sel_idx), _ptr(n_sel), _ptr(inv_idx), _ptr(ws), ws.numel() * ws.element_size(),
                                  _stream()), "vardrop_select")
+
+
+def vardrop_select_static(keys, cfg: SelectCfg, group_id, group_offsets, members, n_groups, sel_idx, n_sel, inv_idx) -> None:
+    """vardrop_select for callers that cannot allocate: no workspace argument, the scratch is a fixed array inside the
+    library (S * N <= 16384).  Calls whose GPU work overlaps share that array and race."""
+    _check(load().vardrop_select_static(_ptr(keys), C.byref(cfg), _ptr(group_id), _ptr(group_offsets), _ptr(members),
+                                        _ptr(n_groups), _ptr(sel_idx), _ptr(n_sel), _ptr(inv_idx), _stream()),
+           "vardrop_select_static")
 
 
 def vardrop_attn_fwd(q, k, v, sel_idx, n_sel, cfg: AttnCfg, o, lse, ws) -> None:

@@ -34,6 +34,12 @@ int select_validate(const vardrop_select_cfg& cfg);
 int select_launch(const uint64_t* keys, const vardrop_select_cfg& cfg, int32_t* group_id, int32_t* group_offsets, int32_t* members,
                   int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, void* ws, cudaStream_t stream);
 
+// allocation-free variant: scratch is a fixed array inside the module
+constexpr int kStaticMaxRows = 16384;                 // largest S * N it accepts
+constexpr int kStaticSelectBytes = 400 * 1024;        // size of that array
+int select_static_launch(const uint64_t* keys, const vardrop_select_cfg& cfg, int32_t* group_id, int32_t* group_offsets,
+                         int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, cudaStream_t stream);
+
 // attn_*.cu
 size_t attn_workspace_bytes(const vardrop_attn_cfg& cfg);
 int attn_validate(const vardrop_attn_cfg& cfg);

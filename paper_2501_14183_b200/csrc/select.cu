@@ -9,6 +9,8 @@
 // Launch 2 (rank in group + finish-by-last-CTA): every member counts the members of its own group with a
 // smaller (priority, rank) pair; it is kept when that count is below the group's quota.  The last CTA of a
 // hash row compacts the kept variates into sel_idx / inv_idx with one scan.
+#include <mutex>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -246,6 +248,41 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
     const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
     { LaunchScope ls_(K_SELECT_SAMPLE, stream); select_sample_kernel<<<grid2, kSelThreads, 0, stream>>>(P); }
     return check_cuda(cudaGetLastError(), "select: sample launch");
+}
+
+// ---- allocation-free variant ------------------------------------------------------------------------------
+// Scratch for vardrop_select_static: a fixed array that is part of the loaded module, so a caller that may not
+// allocate device memory still has somewhere for the counters, ranks, priorities and keep flags to live.
+// Sized for S * N <= kStaticMaxRows (worst case S = kStaticMaxRows, N = 1).
+static __device__ __align__(256) unsigned char g_select_static_scratch[kStaticSelectBytes];
+
+int select_static_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* group_id, int32_t* group_offsets, int32_t* members,
+                         int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, cudaStream_t stream) {
+    if (static_cast<long long>(c.S) * c.N > kStaticMaxRows)
+        return fail(VARDROP_ERR_UNSUPPORTED, "select_static: S*N = %lld exceeds the built-in scratch limit of %d; use vardrop_select with a workspace",
+                    static_cast<long long>(c.S) * c.N, kStaticMaxRows);
+    if (select_workspace_bytes(c) > static_cast<size_t>(kStaticSelectBytes))
+        return fail(VARDROP_ERR_UNSUPPORTED, "select_static: layout of %zu bytes exceeds the built-in scratch of %d bytes",
+                    select_workspace_bytes(c), kStaticSelectBytes);
+    // The array's name is only a handle on the host; the device address is looked up once per device, with that
+    // device current, and remembered.
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* dev_ptr[kMaxDevices] = {};
+    int dev = -1;
+    if (int st = check_cuda(cudaGetDevice(&dev), "select_static: cudaGetDevice")) return st;
+    if (dev < 0 || dev >= kMaxDevices) return fail(VARDROP_ERR_UNSUPPORTED, "select_static: device ordinal %d not supported", dev);
+    void* ptr = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!dev_ptr[dev]) {
+            void* p = nullptr;
+            if (int st = check_cuda(cudaGetSymbolAddress(&p, g_select_static_scratch), "select_static: cudaGetSymbolAddress")) return st;
+            dev_ptr[dev] = p;
+        }
+        ptr = dev_ptr[dev];
+    }
+    return select_launch(keys, c, group_id, group_offsets, members, n_groups, sel_idx, n_sel, inv_idx, ptr, stream);
 }
 
 }  // namespace vardrop

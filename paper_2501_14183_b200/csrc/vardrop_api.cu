@@ -168,6 +168,22 @@ int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t*
                          static_cast<cudaStream_t>(stream));
 }
 
+int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t* group_id, int32_t* group_offsets,
+                          int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(select_validate(*cfg));
+    VD_CHECK(check_ptr(keys, "keys", true));
+    VD_CHECK(check_ptr(group_id, "group_id", true));
+    VD_CHECK(check_ptr(group_offsets, "group_offsets", true));
+    VD_CHECK(check_ptr(members, "members", true));
+    VD_CHECK(check_ptr(n_groups, "n_groups", true));
+    VD_CHECK(check_ptr(sel_idx, "sel_idx", true));
+    VD_CHECK(check_ptr(n_sel, "n_sel", true));
+    VD_CHECK(check_ptr(inv_idx, "inv_idx", true));
+    return select_static_launch(keys, *cfg, group_id, group_offsets, members, n_groups, sel_idx, n_sel, inv_idx,
+                                static_cast<cudaStream_t>(stream));
+}
+
 size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg) {
     if (!cfg || attn_validate(*cfg) != VARDROP_OK) return 0;
     return attn_workspace_bytes(*cfg);
