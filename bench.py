@@ -197,6 +197,7 @@ def kernel_work(w, n_sel):
     kept = w.B * n_sel
     return {
         "hash_kernel": ("hbm", w.B * w.N * w.L * 4 + w.N * (8 + 4 * w.k)),
+        "select_small_kernel": ("hbm", w.N * (8 + 6 * 4)),
         "select_count_kernel": ("hbm", w.N * (8 + 4 * 4)),
         "select_sample_kernel": ("hbm", w.N * 4 * 4),
         "gather_kernel": ("hbm", 2 * 3 * kept * row),

@@ -23,6 +23,11 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
     return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w));
 }
 
+// four consecutive floats added to global memory in one 16-byte reduction
+__device__ __forceinline__ void red_add_f32x4(float* addr, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // prep
 // ---------------------------------------------------------------------------------------------------------
@@ -63,8 +68,10 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
         if (dc == 0) P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + i] = part;
         const size_t dst = (static_cast<size_t>(b) * P.Ncap + i) * chunks_row + c;
         if (P.dog) P.dog[dst] = vd;
-        P.dq_acc[2 * dst] = make_float4(0.f, 0.f, 0.f, 0.f);
-        P.dq_acc[2 * dst + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (n_sel > kTile) {                          // a single key tile writes dq directly, nothing to accumulate
+            P.dq_acc[2 * dst] = make_float4(0.f, 0.f, 0.f, 0.f);
+            P.dq_acc[2 * dst + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
     }
 }
 
@@ -75,12 +82,13 @@ struct BwdParams {
     const float* lse;       // [B, H, N]
     const float* delta;     // [B, H, Ncap]
     float* dq_acc;          // [B, Ncap, H, 64]
-    __nv_bfloat16* dk;      // [B, N, H, D]
+    __nv_bfloat16* dq;      // [B, N, H, D]; written here only when there is a single key tile
+    __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     const int32_t* sel_idx; // NULL: identity
     const int32_t* n_sel;   // NULL: N
     int* status;
-    int N, Ncap, H, D;
+    int B, N, Ncap, H, D;
     float scale, scale_log2;
 };
 
@@ -105,9 +113,9 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
                                                                 const __grid_constant__ CUtensorMap map_v,
                                                                 const __grid_constant__ CUtensorMap map_do, const BwdParams P) {
     const int n_sel = P.n_sel ? *P.n_sel : P.N;
-    const int jt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    if (jt * kTile >= n_sel) return;
-    const int n_q = (n_sel + kTile - 1) / kTile;
+    const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles
+    const int n_items = n_q * P.H * P.B;                       // work items: (key tile, head, instance)
+    if (static_cast<int>(blockIdx.x) >= n_items) return;
 
     extern __shared__ unsigned char smem_dyn[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
@@ -160,130 +168,163 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major, B MN-major, N = 64
     constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_kv, 2 * kTileBytes);
-        tma_load_4d(sK, &map_k, bar_kv, 0, h, jt * kTile, b);
-        tma_load_4d(sV, &map_v, bar_kv, 0, h, jt * kTile, b);
-    }
-    const int key = jt * kTile + tid;               // this thread's key row
-    const bool key_valid = key < n_sel;
     bool ok = true;
+    uint32_t q_count = 0;       // query tiles consumed so far by this CTA (phase of bar_qdo / bar_s / bar_g)
+    uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
+    const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
 
-    for (int i = 0; i < n_q; ++i) {
-        if (tid == 0) {                              // sQ / sdO were released by the wait on bar_g of tile i-1
-            mbar_expect_tx(bar_qdo, 2 * kTileBytes);
-            tma_load_4d(sQ, &map_q, bar_qdo, 0, h, i * kTile, b);
-            tma_load_4d(sdO, &map_do, bar_qdo, 0, h, i * kTile, b);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
+        const int jt = item % n_q;
+        const int h = (item / n_q) % P.H;
+        const int b = item / (n_q * P.H);
+        if (tid == 0) {             // every MMA of the previous item has completed: K and V are free
+            mbar_expect_tx(bar_kv, 2 * kTileBytes);
+            tma_load_4d(sK, &map_k, bar_kv, 0, h, jt * kTile, b);
+            tma_load_4d(sV, &map_v, bar_kv, 0, h, jt * kTile, b);
         }
-        {
-            const int qrow = i * kTile + tid;
-            const bool qv = qrow < n_sel;
-            s_lse[tid] = qv ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
-            s_delta[tid] = qv ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
-        }
-        if (tid == 0) {
-            if (i == 0) ok &= mbar_wait(bar_kv, 0);
-            ok &= mbar_wait(bar_qdo, i & 1);
-            tc_fence_after();
-            const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ), d0 = smem_u32(sdO);
-#pragma unroll
-            for (int ks = 0; ks < kDP / 16; ++ks)
-                tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < kDP / 16; ++ks)
-                tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
-            tc_commit(bar_s);
-        }
-        __syncthreads();                             // row statistics visible
-        ok &= mbar_wait(bar_s, i & 1);
-        tc_fence_after();
+        const int key = jt * kTile + tid;               // this thread's key row
+        const bool key_valid = key < n_sel;
 
-        // ---- P^T and dS^T of this thread's key row over the 128 queries of the tile --------------------------
-        float sv[32], dp[32];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tm_st + lane_sel + c * 32, sv);
-            tmem_ld32(tm_dpt + lane_sel + c * 32, dp);
-            tmem_ld_wait();
-#pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                const int col = c * 32 + x;
-                const float p = key_valid ? exp2f(fmaf(sv[x], P.scale_log2, -s_lse[col])) : 0.f;
-                sv[x] = p;
-                dp[x] = p * (dp[x] - s_delta[col]);
+        for (int i = 0; i < n_q; ++i, ++q_count) {
+            const uint32_t ph = q_count & 1;
+            if (tid == 0) {                              // sQ / sdO were released by the wait on bar_g of the previous tile
+                mbar_expect_tx(bar_qdo, 2 * kTileBytes);
+                tma_load_4d(sQ, &map_q, bar_qdo, 0, h, i * kTile, b);
+                tma_load_4d(sdO, &map_do, bar_qdo, 0, h, i * kTile, b);
             }
-            store_chunk32(sPt, tid, c * 32, sv);
-            store_chunk32(sdSt, tid, c * 32, dp);
-        }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+            {
+                const int qrow = i * kTile + tid;
+                const bool qv = qrow < n_sel;
+                s_lse[tid] = qv ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
+                s_delta[tid] = qv ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
+            }
+            if (tid == 0) {
+                if (i == 0) ok &= mbar_wait(bar_kv, n_done & 1);
+                ok &= mbar_wait(bar_qdo, ph);
+                tc_fence_after();
+                const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ), d0 = smem_u32(sdO);
+#pragma unroll
+                for (int ks = 0; ks < kDP / 16; ++ks)
+                    tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < kDP / 16; ++ks)
+                    tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+                tc_commit(bar_s);
+            }
+            __syncthreads();                             // row statistics visible
+            ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
-            const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ), d0 = smem_u32(sdO), k0 = smem_u32(sK);
+
+            // ---- P^T and dS^T of this thread's key row over the 128 queries of the tile ----------------------
+            float sv[32], dp[32];
 #pragma unroll
-            for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
-                const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
-                tc_mma_bf16(tm_dv, umma_desc_sw128(pt + a_off, 16, 1024), umma_desc_sw128(d0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
-                            (i > 0) | (ks > 0));
-                tc_mma_bf16(tm_dk, umma_desc_sw128(dst + a_off, 16, 1024), umma_desc_sw128(q0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
-                            (i > 0) | (ks > 0));
+            for (int c = 0; c < 4; ++c) {
+                tmem_ld32(tm_st + lane_sel + c * 32, sv);
+                tmem_ld32(tm_dpt + lane_sel + c * 32, dp);
+                tmem_ld_wait();
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    const int col = c * 32 + x;
+                    const float p = key_valid ? exp2f(fmaf(sv[x], P.scale_log2, -s_lse[col])) : 0.f;
+                    sv[x] = p;
+                    dp[x] = p * (dp[x] - s_delta[col]);
+                }
+                store_chunk32(sPt, tid, c * 32, sv);
+                store_chunk32(sdSt, tid, c * 32, dp);
             }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ), d0 = smem_u32(sdO), k0 = smem_u32(sK);
 #pragma unroll
-            for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K
-                tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
-                            idesc_mnmn, ks > 0);
-            tc_commit(bar_g);
+                for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
+                    const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
+                    tc_mma_bf16(tm_dv, umma_desc_sw128(pt + a_off, 16, 1024), umma_desc_sw128(d0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
+                                (i > 0) | (ks > 0));
+                    tc_mma_bf16(tm_dk, umma_desc_sw128(dst + a_off, 16, 1024), umma_desc_sw128(q0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
+                                (i > 0) | (ks > 0));
+                }
+#pragma unroll
+                for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K
+                    tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
+                                idesc_mnmn, ks > 0);
+                tc_commit(bar_g);
+            }
+            ok &= mbar_wait(bar_g, ph);
+            tc_fence_after();
+            {
+                const int qrow = i * kTile + tid;        // tensor-memory lane = query row of dQ_i
+                const bool qv = qrow < n_sel;
+                if (single_tile) {                       // final value: straight to the full-layout gradient, scaled, bf16
+                    const int n = qv ? (P.sel_idx ? P.sel_idx[qrow] : qrow) : 0;
+                    __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
+#pragma unroll
+                    for (int c = 0; c < kDP / 32; ++c) {
+                        if (c * 32 < P.D) {
+                            tmem_ld32(tm_dq + lane_sel + c * 32, sv);
+                            tmem_ld_wait();
+                            if (qv) {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    *reinterpret_cast<uint4*>(dst + c * 32 + q * 8) =
+                                        make_uint4(pack2(sv[8 * q + 0] * P.scale, sv[8 * q + 1] * P.scale), pack2(sv[8 * q + 2] * P.scale, sv[8 * q + 3] * P.scale),
+                                                   pack2(sv[8 * q + 4] * P.scale, sv[8 * q + 5] * P.scale), pack2(sv[8 * q + 6] * P.scale, sv[8 * q + 7] * P.scale));
+                            }
+                        }
+                    }
+                } else {
+                    float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP;
+#pragma unroll
+                    for (int c = 0; c < kDP / 32; ++c) {
+                        tmem_ld32(tm_dq + lane_sel + c * 32, sv);
+                        tmem_ld_wait();
+                        if (qv) {
+#pragma unroll
+                            for (int x = 0; x < 32; x += 4) red_add_f32x4(dst + c * 32 + x, sv[x], sv[x + 1], sv[x + 2], sv[x + 3]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            ok = __syncthreads_and(ok);
+            if (!ok) break;
         }
-        ok &= mbar_wait(bar_g, i & 1);
-        tc_fence_after();
-        {
-            const int qrow = i * kTile + tid;        // tensor-memory lane = query row of dQ_i
-            float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP;
+
+        {   // tensor-memory loads are warp-collective: every thread takes part, only valid key rows store
+            const bool store = ok && key_valid;
+            const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
+            const size_t row = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
+            float acc[32];
 #pragma unroll
             for (int c = 0; c < kDP / 32; ++c) {
-                tmem_ld32(tm_dq + lane_sel + c * 32, sv);
-                tmem_ld_wait();
-                if (qrow < n_sel) {
+                if (c * 32 < P.D) {
+                    tmem_ld32(tm_dv + lane_sel + c * 32, acc);
+                    tmem_ld_wait();
+                    if (store) {
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) atomicAdd(dst + c * 32 + x, sv[x]);
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4*>(P.dv + row + c * 32 + q * 8) =
+                                make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
+                                           pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
+                    }
+                    tmem_ld32(tm_dk + lane_sel + c * 32, acc);
+                    tmem_ld_wait();
+                    if (store) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4*>(P.dk + row + c * 32 + q * 8) =
+                                make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
+                                           pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
+                    }
                 }
             }
+            tc_fence_before();
+            __syncthreads();        // the accumulators are read out before the next item's products overwrite them
         }
-        tc_fence_before();
-        if (!__syncthreads_and(ok)) break;
     }
-
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
-    {   // tensor-memory loads are warp-collective: every thread takes part, only valid key rows store
-        const bool store = ok && key_valid;
-        const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
-        const size_t row = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
-        float acc[32];
-#pragma unroll
-        for (int c = 0; c < kDP / 32; ++c) {
-            if (c * 32 < P.D) {
-                tmem_ld32(tm_dv + lane_sel + c * 32, acc);
-                tmem_ld_wait();
-                if (store) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4*>(P.dv + row + c * 32 + q * 8) =
-                            make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
-                                       pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
-                }
-                tmem_ld32(tm_dk + lane_sel + c * 32, acc);
-                tmem_ld_wait();
-                if (store) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4*>(P.dk + row + c * 32 + q * 8) =
-                            make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
-                                       pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
-                }
-            }
-        }
-    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
@@ -296,12 +337,14 @@ struct FinishParams {
     const float4* dq_acc;    // [B, Ncap, H, 64] fp32
     uint4 *dq, *dk, *dv;     // [B, N, H, D] bf16
     const int32_t* inv_idx;  // NULL: identity
+    const int32_t* n_sel;    // NULL: N
     int N, Ncap, H, D;
     float scale;
 };
 
 __global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
     const int b = blockIdx.y;
+    const bool dq_done = (P.n_sel ? *P.n_sel : P.N) <= kTile;     // single key tile: the main kernel wrote the kept dq rows
     const int chunks_head = P.D / 8;
     const int chunks_row = P.H * chunks_head;
     const int total = P.N * chunks_row;
@@ -312,6 +355,7 @@ __global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
         const int j = P.inv_idx ? P.inv_idx[n] : n;
         const size_t dst = static_cast<size_t>(b) * total + idx;
         if (j >= 0) {
+            if (dq_done) continue;
             const float4* src = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * (kDP / 4) + dc * 2;
             const float4 a = __ldcg(src), c2 = __ldcg(src + 1);
             P.dq[dst] = make_uint4(pack2(a.x * P.scale, a.y * P.scale), pack2(a.z * P.scale, a.w * P.scale),
@@ -345,7 +389,8 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     {
         const long long work = static_cast<long long>(w.Ncap) * c.H * 8;
         int gx = static_cast<int>((work + 255) / 256);
-        if (gx > 1184) gx = 1184;
+        const int cap = max(1, 4 * sm_count() / c.B);              // about four CTAs per SM in total
+        if (gx > cap) gx = cap;
         { LaunchScope ls_(K_BWD_PREP, stream); bwd_prep_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(R); }
         if (int st = check_cuda(cudaGetLastError(), "attention: backward prep launch")) return st;
     }
@@ -364,10 +409,10 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     }
     BwdParams P{};
     P.lse = lse; P.delta = R.delta; P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
-    P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
+    P.dq = static_cast<__nv_bfloat16*>(dq); P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
     P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);
-    P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
+    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
     P.scale = scale; P.scale_log2 = scale * 1.4426950408889634f;
     static thread_local int attr_dev = -1;
     int dev = 0;
@@ -376,18 +421,25 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         if (int st = check_cuda(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
-    { LaunchScope ls_(K_ATTN_BWD, stream); attn_bwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P); }
+    {
+        const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
+        const int grid = static_cast<int>(worst < sm_count() ? worst : sm_count());      // one CTA per SM (all of tensor memory)
+        LaunchScope ls_(K_ATTN_BWD, stream);
+        attn_bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P);
+    }
     if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
 
     FinishParams F{};
     F.dq_acc = reinterpret_cast<const float4*>(base + w.dq_acc);
     F.dq = static_cast<uint4*>(dq); F.dk = static_cast<uint4*>(dk); F.dv = static_cast<uint4*>(dv);
     F.inv_idx = sel_idx ? inv_idx : nullptr;
+    F.n_sel = sel_idx ? n_sel : nullptr;
     F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.scale = scale;
     {
         const long long work = static_cast<long long>(c.N) * c.H * (c.D / 8);
         int gx = static_cast<int>((work + 255) / 256);
-        if (gx > 1184) gx = 1184;
+        const int cap = max(1, 8 * sm_count() / c.B);
+        if (gx > cap) gx = cap;
         { LaunchScope ls_(K_BWD_FINISH, stream); bwd_finish_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F); }
     }
     return check_cuda(cudaGetLastError(), "attention: backward finish launch");

@@ -39,6 +39,9 @@ inline AttnWs attn_layout(const vardrop_attn_cfg& c) {
 // Tensor map over a [B, tokens, H, 64] bf16 tensor: box = one (b, h) tile of 128 tokens x 64 elements,
 // 128-byte swizzle, out-of-range rows read as zero.  `tokens` is the extent the copy engine may touch,
 // `token_stride` the allocated tokens per instance.
+// Number of SMs of the current device (cached per thread and device).
+int sm_count();
+
 int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int token_stride, int H);
 
 // First 1024-byte boundary at or after p (swizzled tiles need it).

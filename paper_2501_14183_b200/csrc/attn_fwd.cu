@@ -29,6 +29,17 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+int sm_count() {
+    static thread_local int cached_dev = -1, cached = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) cached = n;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
 int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int token_stride, int H) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
@@ -97,7 +108,7 @@ struct FwdParams {
     float* lse;
     const int32_t* n_sel;   // NULL: all N tokens
     int* status;
-    int N, H, D;
+    int B, N, H, D;
     float scale_log2;       // sm_scale * log2(e)
 };
 
@@ -127,9 +138,9 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                                                                 const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v, const FwdParams P) {
     const int n_sel = P.n_sel ? *P.n_sel : P.N;
-    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    if (qt * kTile >= n_sel) return;
-    const int n_kv = (n_sel + kTile - 1) / kTile;
+    const int n_kv = (n_sel + kTile - 1) / kTile;              // key tiles = query tiles
+    const int n_items = n_kv * P.H * P.B;                      // work items: (query tile, head, instance)
+    if (static_cast<int>(blockIdx.x) >= n_items) return;
 
     extern __shared__ unsigned char smem_dyn[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);     // barriers and the TMEM slot sit in front of the tiles
@@ -174,114 +185,126 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
     constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
     constexpr uint32_t idesc_o = umma_idesc_bf16(128, kDP, 0, 1);
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, kTileBytes);
-        tma_load_4d(sQ, &map_q, bar_q, 0, h, qt * kTile, b);
-        mbar_expect_tx(bar_kv, 2 * kTileBytes);
-        tma_load_4d(sK, &map_k, bar_kv, 0, h, 0, b);
-        tma_load_4d(sV, &map_v, bar_kv, 0, h, 0, b);
-    }
-
-    float o_acc[kDP];
-#pragma unroll
-    for (int d = 0; d < kDP; ++d) o_acc[d] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
+    uint32_t kv_count = 0;      // K/V tiles consumed so far by this CTA: ring stage and barrier phase follow from it
+    uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_q)
 
-    for (int j = 0; j < n_kv; ++j) {
-        const int st = j & 1;
-        if (tid == 0) {
-            if (j + 1 < n_kv) {                      // the other stage was released by the wait on bar_o of tile j-1
-                mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
-                tma_load_4d(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
-                tma_load_4d(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
+        const int qt = item % n_kv;
+        const int h = (item / n_kv) % P.H;
+        const int b = item / (n_kv * P.H);
+        if (tid == 0) {             // every MMA of the previous item has completed: Q and both ring stages are free
+            mbar_expect_tx(bar_q, kTileBytes);
+            tma_load_4d(sQ, &map_q, bar_q, 0, h, qt * kTile, b);
+            const uint32_t st0 = kv_count & 1;
+            mbar_expect_tx(bar_kv + st0, 2 * kTileBytes);
+            tma_load_4d(sK + st0 * kTileBytes, &map_k, bar_kv + st0, 0, h, 0, b);
+            tma_load_4d(sV + st0 * kTileBytes, &map_v, bar_kv + st0, 0, h, 0, b);
+        }
+
+        float o_acc[kDP];
+#pragma unroll
+        for (int d = 0; d < kDP; ++d) o_acc[d] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;
+
+        for (int j = 0; j < n_kv; ++j, ++kv_count) {
+            const uint32_t st = kv_count & 1;
+            const uint32_t ph = kv_count & 1;            // bar_s / bar_o complete once per key tile
+            if (tid == 0) {
+                if (j + 1 < n_kv) {                      // the other stage was released by the wait on bar_o of the previous tile
+                    mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
+                    tma_load_4d(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
+                    tma_load_4d(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
+                }
+                if (j == 0) ok &= mbar_wait(bar_q, n_done & 1);
+                ok &= mbar_wait(bar_kv + st, (kv_count >> 1) & 1);
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(sK + st * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < kDP / 16; ++ks)
+                    tc_mma_bf16(tmem_s, umma_desc_sw128(a0 + ks * 32, 16, 1024), umma_desc_sw128(b0 + ks * 32, 16, 1024), idesc_s, ks > 0);
+                tc_commit(bar_s);
             }
-            if (j == 0) ok &= mbar_wait(bar_q, 0);
-            ok &= mbar_wait(bar_kv + st, (j >> 1) & 1);
+            ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
-            const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(sK + st * kTileBytes);
-#pragma unroll
-            for (int ks = 0; ks < kDP / 16; ++ks)
-                tc_mma_bf16(tmem_s, umma_desc_sw128(a0 + ks * 32, 16, 1024), umma_desc_sw128(b0 + ks * 32, 16, 1024), idesc_s, ks > 0);
-            tc_commit(bar_s);
-        }
-        ok &= mbar_wait(bar_s, j & 1);
-        tc_fence_after();
 
-        // ---- online softmax of this thread's query row over the 128 keys of the tile ----------------------
-        const int valid = min(kTile, n_sel - j * kTile);      // keys of this tile that exist
-        float s[32];
-        float m_tile = -INFINITY;
+            // ---- online softmax of this thread's query row over the 128 keys of the tile ------------------
+            const int valid = min(kTile, n_sel - j * kTile);      // keys of this tile that exist
+            float s[32];
+            float m_tile = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_s + lane_sel + c * 32, s);
-            tmem_ld_wait();
+            for (int c = 0; c < 4; ++c) {
+                tmem_ld32(tmem_s + lane_sel + c * 32, s);
+                tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (c * 32 + i < valid) m_tile = fmaxf(m_tile, s[i]);
-        }
-        const float m_new = fmaxf(m_run, m_tile * P.scale_log2);
-        const float alpha = exp2f(m_run - m_new);
-        float l_tile = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_s + lane_sel + c * 32, s);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float p = (c * 32 + i < valid) ? exp2f(fmaf(s[i], P.scale_log2, -m_new)) : 0.f;
-                s[i] = p;
-                l_tile += p;
+                for (int i = 0; i < 32; ++i)
+                    if (c * 32 + i < valid) m_tile = fmaxf(m_tile, s[i]);
             }
-            store_row_chunk32(sP, tid, c * 32, s);
-        }
-        l_run = l_run * alpha + l_tile;
-        m_run = m_new;
+            const float m_new = fmaxf(m_run, m_tile * P.scale_log2);
+            const float alpha = exp2f(m_run - m_new);
+            float l_tile = 0.f;
 #pragma unroll
-        for (int d = 0; d < kDP; ++d) o_acc[d] *= alpha;
+            for (int c = 0; c < 4; ++c) {
+                tmem_ld32(tmem_s + lane_sel + c * 32, s);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float p = (c * 32 + i < valid) ? exp2f(fmaf(s[i], P.scale_log2, -m_new)) : 0.f;
+                    s[i] = p;
+                    l_tile += p;
+                }
+                store_row_chunk32(sP, tid, c * 32, s);
+            }
+            l_run = l_run * alpha + l_tile;
+            m_run = m_new;
+#pragma unroll
+            for (int d = 0; d < kDP; ++d) o_acc[d] *= alpha;
 
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(sP), b0 = smem_u32(sV + st * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < kTile / 16; ++ks)
+                    tc_mma_bf16(tmem_o, umma_desc_sw128(a0 + (ks >> 2) * kTileBytes + (ks & 3) * 32, 16, 1024),
+                                umma_desc_sw128(b0 + ks * 2048, kTileBytes, 1024), idesc_o, ks > 0);
+                tc_commit(bar_o);
+            }
+            ok &= mbar_wait(bar_o, ph);
             tc_fence_after();
-            const uint32_t a0 = smem_u32(sP), b0 = smem_u32(sV + st * kTileBytes);
 #pragma unroll
-            for (int ks = 0; ks < kTile / 16; ++ks)
-                tc_mma_bf16(tmem_o, umma_desc_sw128(a0 + (ks >> 2) * kTileBytes + (ks & 3) * 32, 16, 1024),
-                            umma_desc_sw128(b0 + ks * 2048, kTileBytes, 1024), idesc_o, ks > 0);
-            tc_commit(bar_o);
+            for (int c = 0; c < kDP / 32; ++c) {
+                tmem_ld32(tmem_o + lane_sel + c * 32, s);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o_acc[c * 32 + i] += s[i];
+            }
+            tc_fence_before();
+            ok = __syncthreads_and(ok);                  // a wait gave up somewhere in the CTA: stop issuing work
+            if (!ok) break;
         }
-        ok &= mbar_wait(bar_o, j & 1);
-        tc_fence_after();
+
+        const int row = qt * kTile + tid;
+        if (ok && row < n_sel) {
+            const float inv_l = 1.f / l_run;
+            __nv_bfloat16* dst = P.o + ((static_cast<size_t>(b) * P.N + row) * P.H + h) * P.D;
 #pragma unroll
-        for (int c = 0; c < kDP / 32; ++c) {
-            tmem_ld32(tmem_o + lane_sel + c * 32, s);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o_acc[c * 32 + i] += s[i];
+            for (int q = 0; q < kDP / 8; ++q) {
+                if (q * 8 < P.D) {
+                    const uint4 w = make_uint4(pack_bf16(o_acc[8 * q + 0] * inv_l, o_acc[8 * q + 1] * inv_l),
+                                               pack_bf16(o_acc[8 * q + 2] * inv_l, o_acc[8 * q + 3] * inv_l),
+                                               pack_bf16(o_acc[8 * q + 4] * inv_l, o_acc[8 * q + 5] * inv_l),
+                                               pack_bf16(o_acc[8 * q + 6] * inv_l, o_acc[8 * q + 7] * inv_l));
+                    *reinterpret_cast<uint4*>(dst + 8 * q) = w;
+                }
+            }
+            P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
-        tc_fence_before();
-        if (!__syncthreads_and(ok)) break;           // a wait gave up somewhere in the CTA: stop issuing work
     }
 
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
-    const int row = qt * kTile + tid;
-    if (ok && row < n_sel) {
-        const float inv_l = 1.f / l_run;
-        __nv_bfloat16* dst = P.o + ((static_cast<size_t>(b) * P.N + row) * P.H + h) * P.D;
-#pragma unroll
-        for (int q = 0; q < kDP / 8; ++q) {
-            if (q * 8 < P.D) {
-                const uint4 w = make_uint4(pack_bf16(o_acc[8 * q + 0] * inv_l, o_acc[8 * q + 1] * inv_l),
-                                           pack_bf16(o_acc[8 * q + 2] * inv_l, o_acc[8 * q + 3] * inv_l),
-                                           pack_bf16(o_acc[8 * q + 4] * inv_l, o_acc[8 * q + 5] * inv_l),
-                                           pack_bf16(o_acc[8 * q + 6] * inv_l, o_acc[8 * q + 7] * inv_l));
-                *reinterpret_cast<uint4*>(dst + 8 * q) = w;
-            }
-        }
-        P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kFwdTmemCols);
@@ -305,7 +328,8 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D;
         const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
         int gx = static_cast<int>((work + 255) / 256);
-        if (gx > 1184) gx = 1184;
+        const int cap = max(1, 4 * sm_count() / (3 * c.B));        // about four CTAs per SM in total; each strides over its rows
+        if (gx > cap) gx = cap;
         { LaunchScope ls_(K_GATHER, stream); gather_kernel<<<dim3(gx, c.B, 3), 256, 0, stream>>>(G); }
         if (int st = check_cuda(cudaGetLastError(), "attention: gather launch")) return st;
         if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
@@ -319,7 +343,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
     FwdParams P{};
     P.o = static_cast<__nv_bfloat16*>(o); P.lse = lse; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);
-    P.N = c.N; P.H = c.H; P.D = c.D;
+    P.B = c.B; P.N = c.N; P.H = c.H; P.D = c.D;
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
     P.scale_log2 = scale * 1.4426950408889634f;
     static thread_local int attr_dev = -1;
@@ -329,7 +353,12 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         if (int st = check_cuda(cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
-    { LaunchScope ls_(K_ATTN_FWD, stream); attn_fwd_kernel<<<dim3(w.Ncap / kTile, c.H, c.B), kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P); }
+    {
+        const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
+        const int grid = static_cast<int>(worst < 2ll * sm_count() ? worst : 2ll * sm_count());      // two CTAs fit per SM
+        LaunchScope ls_(K_ATTN_FWD, stream);
+        attn_fwd_kernel<<<grid, kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P);
+    }
     return check_cuda(cudaGetLastError(), "attention: forward launch");
 }
 

@@ -193,6 +193,153 @@ __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const Select
     if (threadIdx.x == 0) P.n_sel[s] = total;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Small problems (N <= 2048): one CTA per hash row does everything in shared memory with two bitonic sorts.
+//   sort 1: (key, variate)                      -> members, group heads -> ids, offsets
+//   sort 2: (group id, Philox priority, rank j) -> position inside the group = sampling rank
+// then the kept flags are compacted with one scan.  No scratch in global memory, no atomics.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kSmallMaxN = 2048;
+
+// Bitonic sort of M (a power of two) items in shared memory by M / 2 threads, one compare-exchange per thread and stage.
+// Items are (key, payload) pairs ordered by key, then payload.
+__device__ __forceinline__ void bitonic_sort_pairs(ulonglong2* a, int M) {
+    const int t = threadIdx.x;
+    for (int k = 2; k <= M; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // lower index of this thread's pair (bit j clear)
+            const int l = i | j;
+            const bool up = (i & k) == 0;
+            const ulonglong2 x = a[i], y = a[l];
+            const bool gt = x.x > y.x || (x.x == y.x && x.y > y.y);
+            if (gt == up) { a[i] = y; a[l] = x; }
+            __syncthreads();
+        }
+    }
+}
+__device__ __forceinline__ void bitonic_sort_u64(uint64_t* a, int M) {
+    const int t = threadIdx.x;
+    for (int k = 2; k <= M; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+            const int l = i | j;
+            const bool up = (i & k) == 0;
+            const uint64_t x = a[i], y = a[l];
+            if ((x > y) == up) { a[i] = y; a[l] = x; }
+            __syncthreads();
+        }
+    }
+}
+
+// exclusive scan of two values per thread (positions 2 tid and 2 tid + 1) over the CTA; returns the exclusive prefix
+// of position 2 tid and the total
+__device__ __forceinline__ int block_scan_pair(int v0, int v1, int* warp_sums, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    int v = v0 + v1;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += o;
+    }
+    __syncthreads();
+    if (lane == 31) warp_sums[warp] = v;
+    __syncthreads();
+    int base = 0, tot = 0;
+    for (int w = 0; w < n_warps; ++w) {
+        const int sw = warp_sums[w];
+        if (w < warp) base += sw;
+        tot += sw;
+    }
+    *total = tot;
+    return v + base - v0 - v1;
+}
+
+// launched with M / 2 threads (M >= 64 a power of two, N <= M)
+__global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const SelectParams P, int M) {
+    extern __shared__ __align__(16) unsigned char sm_raw[];
+    ulonglong2* a2 = reinterpret_cast<ulonglong2*>(sm_raw);       // [M] (key, variate) pairs
+    uint64_t* a = reinterpret_cast<uint64_t*>(a2 + M);            // [M] (group, priority, rank) codes
+    uint32_t* idx = reinterpret_cast<uint32_t*>(a + M);           // [M] variate by sorted position
+    int* gpos = reinterpret_cast<int*>(idx + M);                  // [M] group id by sorted position
+    int* off_s = gpos + M;                                        // [M + 1] group offsets
+    int* keep_s = off_s + M + 1;                                  // [M] kept flag by variate
+    __shared__ int warp_sums[kSmallMaxN / 64];
+    const int s = blockIdx.x, N = P.N, tid = threadIdx.x;
+    const uint64_t* keys = P.keys + static_cast<size_t>(s) * N;
+    int32_t* members = P.members + static_cast<size_t>(s) * N;
+    int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
+    int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
+    int32_t* sel = P.sel_idx + static_cast<size_t>(s) * N;
+    int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
+    const int p0 = 2 * tid, p1 = 2 * tid + 1;                     // the two positions this thread owns outside the sorts
+
+    if (s == 0 && tid == 0) *P.status = VARDROP_OK;               // nothing in this kernel can fail on the device
+    a2[p0] = make_ulonglong2(p0 < N ? keys[p0] : ~0ull, static_cast<uint64_t>(p0));
+    a2[p1] = make_ulonglong2(p1 < N ? keys[p1] : ~0ull, static_cast<uint64_t>(p1));
+    __syncthreads();
+    bitonic_sort_pairs(a2, M);
+
+    // group heads -> dense ids and offsets
+    const int h0 = (p0 < N) && (p0 == 0 || a2[p0].x != a2[p0 - 1].x);
+    const int h1 = (p1 < N) && (a2[p1].x != a2[p1 - 1].x);
+    int G = 0;
+    const int before = block_scan_pair(h0, h1, warp_sums, &G);
+    if (p0 < N) {
+        const int g = before + h0 - 1, n = static_cast<int>(a2[p0].y);
+        gpos[p0] = g; idx[p0] = n;
+        if (h0) { off_s[g] = p0; off[g] = p0; }
+        members[p0] = n;
+        gid[n] = g;
+    }
+    if (p1 < N) {
+        const int g = before + h0 + h1 - 1, n = static_cast<int>(a2[p1].y);
+        gpos[p1] = g; idx[p1] = n;
+        if (h1) { off_s[g] = p1; off[g] = p1; }
+        members[p1] = n;
+        gid[n] = g;
+    }
+    if (tid == 0) { off_s[G] = N; P.n_groups[s] = G; }
+    for (int i = G + tid; i <= N; i += blockDim.x) off[i] = N;
+    __syncthreads();
+
+    // sampling rank: sort (group, priority, j)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int p = 2 * tid + e;
+        uint64_t c = ~0ull;
+        if (p < N) {
+            const int g = gpos[p];
+            const int j = p - off_s[g];
+            const uint32_t pri = philox4x32_10_word0(static_cast<uint32_t>(j), static_cast<uint32_t>(g), static_cast<uint32_t>(s), P.step,
+                                                     P.seed_lo, P.seed_hi);
+            c = (static_cast<uint64_t>(g) << 43) | (static_cast<uint64_t>(pri) << 11) | static_cast<uint64_t>(j);
+        }
+        a[p] = c;
+    }
+    __syncthreads();
+    bitonic_sort_u64(a, M);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int q = 2 * tid + e;
+        if (q < N) {
+            const uint64_t c = a[q];
+            const int g = static_cast<int>(c >> 43), j = static_cast<int>(c & 2047u);
+            const int begin = off_s[g], size = off_s[g + 1] - begin;
+            keep_s[idx[begin + j]] = (q - begin) < quota_of(size, P.gs, P.rate_ppm);
+        }
+    }
+    __syncthreads();
+
+    // compaction in ascending variate order
+    const int k0 = p0 < N ? keep_s[p0] : 0, k1 = p1 < N ? keep_s[p1] : 0;
+    int total = 0;
+    int pos = block_scan_pair(k0, k1, warp_sums, &total);
+    if (p0 < N) { if (k0) { sel[pos] = p0; inv[p0] = pos; ++pos; } else inv[p0] = -1; }
+    if (p1 < N) { if (k1) { sel[pos] = p1; inv[p1] = pos; } else inv[p1] = -1; }
+    for (int i = total + tid; i < N; i += blockDim.x) sel[i] = -1;
+    if (tid == 0) P.n_sel[s] = total;
+}
+
 struct SelectWs {
     size_t done1, done2, lt, eq, prio, keep, total, zero_begin, zero_bytes;
 };
@@ -241,6 +388,20 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
     P.seed_lo = static_cast<uint32_t>(c.seed & 0xFFFFFFFFu);
     P.seed_hi = static_cast<uint32_t>(c.seed >> 32);
     P.step = c.step;
+    if (c.N <= kSmallMaxN) {
+        int M = 64;
+        while (M < c.N) M <<= 1;
+        const size_t smem = static_cast<size_t>(M) * (16 + 8 + 4 + 4 + 4 + 4) + 16;
+        static thread_local int attr_dev = -1;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (attr_dev != dev) {
+            if (int st = check_cuda(cudaFuncSetAttribute(select_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024), "select: smem attribute")) return st;
+            attr_dev = dev;
+        }
+        { LaunchScope ls_(K_SELECT_SMALL, stream); select_small_kernel<<<c.S, M / 2, smem, stream>>>(P, M); }
+        return check_cuda(cudaGetLastError(), "select: launch");
+    }
     if (int st = check_cuda(cudaMemsetAsync(base, 0, w.zero_begin + w.zero_bytes, stream), "select: clear counters")) return st;
     const dim3 grid1((c.N + kSelThreads - 1) / kSelThreads, (c.N + kKeyChunk - 1) / kKeyChunk, c.S);
     { LaunchScope ls_(K_SELECT_COUNT, stream); select_count_kernel<<<grid1, kSelThreads, 0, stream>>>(P); }
