@@ -92,11 +92,19 @@ struct BwdParams {
     float scale, scale_log2;
 };
 
-constexpr int kBwdThreads = 128;
+constexpr int kBwdThreads = 256;       // two threads per tensor-memory lane: each takes one 64-column half
 constexpr uint32_t kBwdTmemCols = 512;
-constexpr int kBwdSmemBytes = 2048 /*barriers, row statistics, alignment*/ + 4 * kTileBytes /*K, V, Q, dO*/ + 4 * kTileBytes /*P^T, dS^T*/;
+constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 4 * kTileBytes /*Q, dO x 2 stages*/ +
+                              4 * kTileBytes /*P^T, dS^T*/;
 
-// 32 consecutive columns of row r of a 128 x 128 bf16 tile stored as two 64-column panels (128-byte swizzled rows)
+__device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// 32 consecutive columns (c0 a multiple of 32) of row r of a 128 x 128 bf16 tile stored as two 64-column panels
+// (128-byte swizzled rows)
 __device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0, const float* v) {
     unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
     const int chunk0 = (c0 & 63) >> 3;
@@ -108,10 +116,10 @@ __device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0
     }
 }
 
-__global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
-                                                                const __grid_constant__ CUtensorMap map_k,
-                                                                const __grid_constant__ CUtensorMap map_v,
-                                                                const __grid_constant__ CUtensorMap map_do, const BwdParams P) {
+__global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                   const __grid_constant__ CUtensorMap map_k,
+                                                                   const __grid_constant__ CUtensorMap map_v,
+                                                                   const __grid_constant__ CUtensorMap map_do, const BwdParams P) {
     const int n_sel = P.n_sel ? *P.n_sel : P.N;
     const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles
     const int n_items = n_q * P.H * P.B;                       // work items: (key tile, head, instance)
@@ -120,17 +128,16 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     extern __shared__ unsigned char smem_dyn[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
     uint64_t* bar_kv = bars + 0;
-    uint64_t* bar_qdo = bars + 1;
-    uint64_t* bar_s = bars + 2;
-    uint64_t* bar_g = bars + 3;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
-    float* s_lse = reinterpret_cast<float*>(smem_dyn + 64);       // [128] log2-domain row statistics of the query tile
-    float* s_delta = s_lse + kTile;                               // [128]
-    unsigned char* sK = align_tiles(smem_dyn + 64 + 2 * kTile * sizeof(float));
+    uint64_t* bar_qdo = bars + 1;                   // [2]
+    uint64_t* bar_s = bars + 3;
+    uint64_t* bar_g = bars + 4;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+    float* s_stat = reinterpret_cast<float*>(smem_dyn + 64);      // [2 stages][lse (log2 domain) 128 | Delta 128]
+    unsigned char* sK = align_tiles(smem_dyn + 64 + 4 * kTile * sizeof(float));
     unsigned char* sV = sK + kTileBytes;
-    unsigned char* sQ = sV + kTileBytes;
-    unsigned char* sdO = sQ + kTileBytes;
-    unsigned char* sPt = sdO + kTileBytes;          // P^T  : rows = keys, columns = queries (two 64-query panels)
+    unsigned char* sQ = sV + kTileBytes;            // 2 stages
+    unsigned char* sdO = sQ + 2 * kTileBytes;       // 2 stages
+    unsigned char* sPt = sdO + 2 * kTileBytes;      // P^T  : rows = keys, columns = queries (two 64-query panels)
     unsigned char* sdSt = sPt + 2 * kTileBytes;     // dS^T : same shape
     if (sdSt + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
         if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
@@ -138,13 +145,16 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     }
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int row = tid & (kTile - 1);              // tensor-memory lane this thread reads
+    const int half = tid >> 7;                      // which 64-column half of the lane
     if (warp == 0) {
         tmem_alloc(tmem_slot, kBwdTmemCols);
         tmem_relinquish();
     }
     if (tid == 0) {
         mbar_init(bar_kv, 1);
-        mbar_init(bar_qdo, 1);
+        mbar_init(bar_qdo + 0, 1);
+        mbar_init(bar_qdo + 1, 1);
         mbar_init(bar_s, 1);
         mbar_init(bar_g, 1);
         mbar_fence_init();
@@ -162,47 +172,57 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     const uint32_t tm_dv = tmem + 256;      // [256,320) dV
     const uint32_t tm_dk = tmem + 320;      // [320,384) dK
     const uint32_t tm_dq = tmem + 384;      // [384,448) dQ of the current query tile
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
 
     constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);     // K-major x K-major, N = 128
     constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major, B MN-major, N = 64
     constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
 
     bool ok = true;
-    uint32_t q_count = 0;       // query tiles consumed so far by this CTA (phase of bar_qdo / bar_s / bar_g)
+    uint32_t q_count = 0;       // query tiles consumed so far by this CTA: stage = q_count & 1
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
     const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
+
+    // row statistic of query `qrow`: threads 0..127 fetch lse (log2 domain), threads 128..255 fetch Delta
+    auto load_stat = [&](int b, int h, int qrow) -> float {
+        if (qrow >= n_sel) return half == 0 ? INFINITY : 0.f;
+        return half == 0 ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f
+                         : P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow];
+    };
 
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
         const int jt = item % n_q;
         const int h = (item / n_q) % P.H;
         const int b = item / (n_q * P.H);
-        if (tid == 0) {             // every MMA of the previous item has completed: K and V are free
+        if (tid == 0) {             // every MMA of the previous item has completed: K, V and both Q/dO stages are free
             mbar_expect_tx(bar_kv, 2 * kTileBytes);
             tma_load_4d(sK, &map_k, bar_kv, 0, h, jt * kTile, b);
             tma_load_4d(sV, &map_v, bar_kv, 0, h, jt * kTile, b);
+            const uint32_t st0 = q_count & 1;
+            mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
+            tma_load_4d(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, 0, h, 0, b);
+            tma_load_4d(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, 0, h, 0, b);
         }
-        const int key = jt * kTile + tid;               // this thread's key row
+        s_stat[(q_count & 1) * 2 * kTile + tid] = load_stat(b, h, row);
+        const int key = jt * kTile + row;               // this thread's key row
         const bool key_valid = key < n_sel;
 
         for (int i = 0; i < n_q; ++i, ++q_count) {
-            const uint32_t ph = q_count & 1;
-            if (tid == 0) {                              // sQ / sdO were released by the wait on bar_g of the previous tile
-                mbar_expect_tx(bar_qdo, 2 * kTileBytes);
-                tma_load_4d(sQ, &map_q, bar_qdo, 0, h, i * kTile, b);
-                tma_load_4d(sdO, &map_do, bar_qdo, 0, h, i * kTile, b);
-            }
-            {
-                const int qrow = i * kTile + tid;
-                const bool qv = qrow < n_sel;
-                s_lse[tid] = qv ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
-                s_delta[tid] = qv ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
+            const uint32_t st = q_count & 1, ph = q_count & 1;
+            float next_stat = 0.f;
+            if (i + 1 < n_q) {
+                if (tid == 0) {                          // the other stage was released by the wait on bar_g of the previous tile
+                    mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);
+                    tma_load_4d(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), 0, h, (i + 1) * kTile, b);
+                    tma_load_4d(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), 0, h, (i + 1) * kTile, b);
+                }
+                next_stat = load_stat(b, h, (i + 1) * kTile + row);      // lands while this tile is processed
             }
             if (tid == 0) {
                 if (i == 0) ok &= mbar_wait(bar_kv, n_done & 1);
-                ok &= mbar_wait(bar_qdo, ph);
+                ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
                 tc_fence_after();
-                const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ), d0 = smem_u32(sdO);
+                const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ + st * kTileBytes), d0 = smem_u32(sdO + st * kTileBytes);
 #pragma unroll
                 for (int ks = 0; ks < kDP / 16; ++ks)
                     tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
@@ -211,33 +231,43 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
                     tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
                 tc_commit(bar_s);
             }
-            __syncthreads();                             // row statistics visible
+            __syncthreads();                             // row statistics of this stage visible
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
 
-            // ---- P^T and dS^T of this thread's key row over the 128 queries of the tile ----------------------
-            float sv[32], dp[32];
+            // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
+            const float* lse2 = s_stat + st * 2 * kTile + half * 64;
+            const float* dlt = lse2 + kTile;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(tm_st + lane_sel + c * 32, sv);
-                tmem_ld32(tm_dpt + lane_sel + c * 32, dp);
+            for (int c = 0; c < 2; ++c) {
+                float sv[32], dp[32];
+                tmem_ld32(tm_st + lane_sel + half * 64 + c * 32, sv);
+                tmem_ld32(tm_dpt + lane_sel + half * 64 + c * 32, dp);
                 tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    const int col = c * 32 + x;
-                    const float p = key_valid ? exp2f(fmaf(sv[x], P.scale_log2, -s_lse[col])) : 0.f;
-                    sv[x] = p;
-                    dp[x] = p * (dp[x] - s_delta[col]);
+                for (int x = 0; x < 32; x += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 32 + x);
+                    const float4 d4 = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
+                    const float p0 = fast_exp2(fmaf(sv[x + 0], P.scale_log2, -l4.x)), p1 = fast_exp2(fmaf(sv[x + 1], P.scale_log2, -l4.y));
+                    const float p2 = fast_exp2(fmaf(sv[x + 2], P.scale_log2, -l4.z)), p3 = fast_exp2(fmaf(sv[x + 3], P.scale_log2, -l4.w));
+                    sv[x + 0] = p0; sv[x + 1] = p1; sv[x + 2] = p2; sv[x + 3] = p3;
+                    dp[x + 0] = p0 * (dp[x + 0] - d4.x); dp[x + 1] = p1 * (dp[x + 1] - d4.y);
+                    dp[x + 2] = p2 * (dp[x + 2] - d4.z); dp[x + 3] = p3 * (dp[x + 3] - d4.w);
                 }
-                store_chunk32(sPt, tid, c * 32, sv);
-                store_chunk32(sdSt, tid, c * 32, dp);
+                if (!key_valid) {                        // rows past n_sel hold zero keys: their probabilities must not count
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) { sv[x] = 0.f; dp[x] = 0.f; }
+                }
+                store_chunk32(sPt, row, half * 64 + c * 32, sv);
+                store_chunk32(sdSt, row, half * 64 + c * 32, dp);
             }
             fence_proxy_async_smem();
             tc_fence_before();
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
-                const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ), d0 = smem_u32(sdO), k0 = smem_u32(sK);
+                const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ + st * kTileBytes), d0 = smem_u32(sdO + st * kTileBytes),
+                               k0 = smem_u32(sK);
 #pragma unroll
                 for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
                     const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
@@ -252,39 +282,29 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
                                 idesc_mnmn, ks > 0);
                 tc_commit(bar_g);
             }
+            if (i + 1 < n_q) s_stat[(st ^ 1) * 2 * kTile + tid] = next_stat;      // read only after the next top-of-loop barrier
             ok &= mbar_wait(bar_g, ph);
             tc_fence_after();
-            {
-                const int qrow = i * kTile + tid;        // tensor-memory lane = query row of dQ_i
+            {   // dQ_i: tensor-memory lane = query row; this thread drains 32 of the 64 head-dimension columns
+                const int qrow = i * kTile + row;
                 const bool qv = qrow < n_sel;
+                float dqv[32];
+                tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
+                tmem_ld_wait();
                 if (single_tile) {                       // final value: straight to the full-layout gradient, scaled, bf16
-                    const int n = qv ? (P.sel_idx ? P.sel_idx[qrow] : qrow) : 0;
-                    __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
+                    if (qv && half * 32 < P.D) {
+                        const int n = P.sel_idx ? P.sel_idx[qrow] : qrow;
+                        __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
 #pragma unroll
-                    for (int c = 0; c < kDP / 32; ++c) {
-                        if (c * 32 < P.D) {
-                            tmem_ld32(tm_dq + lane_sel + c * 32, sv);
-                            tmem_ld_wait();
-                            if (qv) {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    *reinterpret_cast<uint4*>(dst + c * 32 + q * 8) =
-                                        make_uint4(pack2(sv[8 * q + 0] * P.scale, sv[8 * q + 1] * P.scale), pack2(sv[8 * q + 2] * P.scale, sv[8 * q + 3] * P.scale),
-                                                   pack2(sv[8 * q + 4] * P.scale, sv[8 * q + 5] * P.scale), pack2(sv[8 * q + 6] * P.scale, sv[8 * q + 7] * P.scale));
-                            }
-                        }
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4*>(dst + q * 8) =
+                                make_uint4(pack2(dqv[8 * q + 0] * P.scale, dqv[8 * q + 1] * P.scale), pack2(dqv[8 * q + 2] * P.scale, dqv[8 * q + 3] * P.scale),
+                                           pack2(dqv[8 * q + 4] * P.scale, dqv[8 * q + 5] * P.scale), pack2(dqv[8 * q + 6] * P.scale, dqv[8 * q + 7] * P.scale));
                     }
-                } else {
-                    float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP;
+                } else if (qv) {
+                    float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP + half * 32;
 #pragma unroll
-                    for (int c = 0; c < kDP / 32; ++c) {
-                        tmem_ld32(tm_dq + lane_sel + c * 32, sv);
-                        tmem_ld_wait();
-                        if (qv) {
-#pragma unroll
-                            for (int x = 0; x < 32; x += 4) red_add_f32x4(dst + c * 32 + x, sv[x], sv[x + 1], sv[x + 2], sv[x + 3]);
-                        }
-                    }
+                    for (int x = 0; x < 32; x += 4) red_add_f32x4(dst + x, dqv[x], dqv[x + 1], dqv[x + 2], dqv[x + 3]);
                 }
             }
             tc_fence_before();
@@ -292,33 +312,28 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
             if (!ok) break;
         }
 
-        {   // tensor-memory loads are warp-collective: every thread takes part, only valid key rows store
-            const bool store = ok && key_valid;
+        {   // dV, dK of this key tile: every thread takes part in the warp-collective loads, only valid key rows store
+            const bool store = ok && key_valid && half * 32 < P.D;
             const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
-            const size_t row = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D;
+            const size_t out = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
             float acc[32];
+            tmem_ld32(tm_dv + lane_sel + half * 32, acc);
+            tmem_ld_wait();
+            if (store) {
 #pragma unroll
-            for (int c = 0; c < kDP / 32; ++c) {
-                if (c * 32 < P.D) {
-                    tmem_ld32(tm_dv + lane_sel + c * 32, acc);
-                    tmem_ld_wait();
-                    if (store) {
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4*>(P.dv + out + q * 8) =
+                        make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
+                                   pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
+            }
+            tmem_ld32(tm_dk + lane_sel + half * 32, acc);
+            tmem_ld_wait();
+            if (store) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4*>(P.dv + row + c * 32 + q * 8) =
-                                make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
-                                           pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
-                    }
-                    tmem_ld32(tm_dk + lane_sel + c * 32, acc);
-                    tmem_ld_wait();
-                    if (store) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4*>(P.dk + row + c * 32 + q * 8) =
-                                make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
-                                           pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
-                    }
-                }
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4*>(P.dk + out + q * 8) =
+                        make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
+                                   pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
             }
             tc_fence_before();
             __syncthreads();        // the accumulators are read out before the next item's products overwrite them

@@ -116,6 +116,13 @@ constexpr int kFwdThreads = 128;
 constexpr uint32_t kFwdTmemCols = 256;
 constexpr int kFwdSmemBytes = 1024 /*barriers + alignment*/ + kTileBytes /*Q*/ + 2 * kTileBytes /*K*/ + 2 * kTileBytes /*V*/ + 2 * kTileBytes /*P*/;
 
+// 2^x by the special-function unit (relative error about 2^-22; -inf gives 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<const uint32_t*>(&v);
@@ -205,7 +212,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
         float o_acc[kDP];
 #pragma unroll
         for (int d = 0; d < kDP; ++d) o_acc[d] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_run = -INFINITY, l_run = 0.f, alpha = 0.f;
 
         for (int j = 0; j < n_kv; ++j, ++kv_count) {
             const uint32_t st = kv_count & 1;
@@ -230,35 +237,33 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
 
             // ---- online softmax of this thread's query row over the 128 keys of the tile ------------------
             const int valid = min(kTile, n_sel - j * kTile);      // keys of this tile that exist
-            float s[32];
-            float m_tile = -INFINITY;
+            float s[kTile];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(tmem_s + lane_sel + c * 32, s);
-                tmem_ld_wait();
+            for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_sel + c * 32, s + c * 32);
+            tmem_ld_wait();
+            if (valid < kTile) {                                  // ragged last tile: keys past n_sel never win the max
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c * 32 + i < valid) m_tile = fmaxf(m_tile, s[i]);
+                for (int i = 0; i < kTile; ++i)
+                    if (i >= valid) s[i] = -INFINITY;
             }
+            float mx[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mx[i] = s[i];
+#pragma unroll
+            for (int i = 8; i < kTile; ++i) mx[i & 7] = fmaxf(mx[i & 7], s[i]);
+            const float m_tile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
             const float m_new = fmaxf(m_run, m_tile * P.scale_log2);
-            const float alpha = exp2f(m_run - m_new);
-            float l_tile = 0.f;
+            alpha = fast_exp2(m_run - m_new);
+            float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(tmem_s + lane_sel + c * 32, s);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float p = (c * 32 + i < valid) ? exp2f(fmaf(s[i], P.scale_log2, -m_new)) : 0.f;
-                    s[i] = p;
-                    l_tile += p;
-                }
-                store_row_chunk32(sP, tid, c * 32, s);
+            for (int i = 0; i < kTile; ++i) {                     // exp2(-inf) = 0 for the masked keys
+                s[i] = fast_exp2(fmaf(s[i], P.scale_log2, -m_new));
+                l4[i & 3] += s[i];
             }
-            l_run = l_run * alpha + l_tile;
-            m_run = m_new;
 #pragma unroll
-            for (int d = 0; d < kDP; ++d) o_acc[d] *= alpha;
+            for (int c = 0; c < 4; ++c) store_row_chunk32(sP, tid, c * 32, s + c * 32);
+            l_run = l_run * alpha + ((l4[0] + l4[1]) + (l4[2] + l4[3]));
+            m_run = m_new;
 
             fence_proxy_async_smem();
             tc_fence_before();
@@ -275,11 +280,13 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
             ok &= mbar_wait(bar_o, ph);
             tc_fence_after();
 #pragma unroll
-            for (int c = 0; c < kDP / 32; ++c) {
-                tmem_ld32(tmem_o + lane_sel + c * 32, s);
+            {
+                float ov[kDP];
+#pragma unroll
+                for (int c = 0; c < kDP / 32; ++c) tmem_ld32(tmem_o + lane_sel + c * 32, ov + c * 32);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o_acc[c * 32 + i] += s[i];
+                for (int d = 0; d < kDP; ++d) o_acc[d] = fmaf(o_acc[d], alpha, ov[d]);     // rescale and add in one step
             }
             tc_fence_before();
             ok = __syncthreads_and(ok);                  // a wait gave up somewhere in the CTA: stop issuing work
