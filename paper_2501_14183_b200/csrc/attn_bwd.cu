@@ -183,6 +183,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
     const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
 
+    // S^T = K Q^T and dP^T = V dO^T of one query tile (issued by one thread), completion on bar_s
+    auto issue_scores = [&](const unsigned char* q_tile, const unsigned char* do_tile) {
+        const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(q_tile), d0 = smem_u32(do_tile);
+#pragma unroll
+        for (int ks = 0; ks < kDP / 16; ++ks)
+            tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < kDP / 16; ++ks)
+            tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+        tc_commit(bar_s);
+    };
+
     // row statistic of query `qrow`: threads 0..127 fetch lse (log2 domain), threads 128..255 fetch Delta
     auto load_stat = [&](int b, int h, int qrow) -> float {
         if (qrow >= n_sel) return half == 0 ? INFINITY : 0.f;
@@ -218,18 +230,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
                 next_stat = load_stat(b, h, (i + 1) * kTile + row);      // lands while this tile is processed
             }
-            if (tid == 0) {
-                if (i == 0) ok &= mbar_wait(bar_kv, n_done & 1);
+            if (tid == 0 && i == 0) {                    // later tiles: issued right behind the previous tile's products
+                ok &= mbar_wait(bar_kv, n_done & 1);
                 ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
                 tc_fence_after();
-                const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(sQ + st * kTileBytes), d0 = smem_u32(sdO + st * kTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < kDP / 16; ++ks)
-                    tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < kDP / 16; ++ks)
-                    tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
-                tc_commit(bar_s);
+                issue_scores(sQ + st * kTileBytes, sdO + st * kTileBytes);
             }
             __syncthreads();                             // row statistics of this stage visible
             ok &= mbar_wait(bar_s, ph);
@@ -281,6 +286,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
                                 idesc_mnmn, ks > 0);
                 tc_commit(bar_g);
+                if (i + 1 < n_q) {                       // S^T, dP^T of the next query tile queue up behind these products
+                    ok &= mbar_wait(bar_qdo + (st ^ 1), ((q_count + 1) >> 1) & 1);
+                    tc_fence_after();
+                    issue_scores(sQ + (st ^ 1) * kTileBytes, sdO + (st ^ 1) * kTileBytes);
+                }
             }
             if (i + 1 < n_q) s_stat[(st ^ 1) * 2 * kTile + tid] = next_stat;      // read only after the next top-of-loop barrier
             ok &= mbar_wait(bar_g, ph);

@@ -185,12 +185,20 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tmem_s = tmem;                   // columns [0, 128): S
-    const uint32_t tmem_o = tmem + 128;             // columns [128, 192): P V of the current key tile
+    // two 128-column buffers: S of tile j lives in buffer j & 1; once the softmax has read it, P V of the same tile
+    // lands in its first 64 columns while S of tile j + 1 is produced in the other buffer
     const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
 
     constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
     constexpr uint32_t idesc_o = umma_idesc_bf16(128, kDP, 0, 1);
+
+    auto issue_scores = [&](uint32_t tmem_dst, const unsigned char* k_tile) {     // S = Q K^T, completion on bar_s
+        const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(k_tile);
+#pragma unroll
+        for (int ks = 0; ks < kDP / 16; ++ks)
+            tc_mma_bf16(tmem_dst, umma_desc_sw128(a0 + ks * 32, 16, 1024), umma_desc_sw128(b0 + ks * 32, 16, 1024), idesc_s, ks > 0);
+        tc_commit(bar_s);
+    };
 
     bool ok = true;
     uint32_t kv_count = 0;      // K/V tiles consumed so far by this CTA: ring stage and barrier phase follow from it
@@ -223,15 +231,15 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                     tma_load_4d(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
                     tma_load_4d(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
                 }
-                if (j == 0) ok &= mbar_wait(bar_q, n_done & 1);
-                ok &= mbar_wait(bar_kv + st, (kv_count >> 1) & 1);
-                tc_fence_after();
-                const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(sK + st * kTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < kDP / 16; ++ks)
-                    tc_mma_bf16(tmem_s, umma_desc_sw128(a0 + ks * 32, 16, 1024), umma_desc_sw128(b0 + ks * 32, 16, 1024), idesc_s, ks > 0);
-                tc_commit(bar_s);
+                if (j == 0) {                            // later tiles: issued right behind the previous tile's P V
+                    ok &= mbar_wait(bar_q, n_done & 1);
+                    ok &= mbar_wait(bar_kv + st, (kv_count >> 1) & 1);
+                    tc_fence_after();
+                    issue_scores(tmem + st * 128, sK + st * kTileBytes);
+                }
             }
+            const uint32_t tmem_s = tmem + st * 128;     // S of this tile; its first 64 columns are reused for P V
+            const uint32_t tmem_o = tmem_s;
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
 
@@ -276,6 +284,11 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                     tc_mma_bf16(tmem_o, umma_desc_sw128(a0 + (ks >> 2) * kTileBytes + (ks & 3) * 32, 16, 1024),
                                 umma_desc_sw128(b0 + ks * 2048, kTileBytes, 1024), idesc_o, ks > 0);
                 tc_commit(bar_o);
+                if (j + 1 < n_kv) {                      // scores of the next key tile queue up behind P V, in the other buffer
+                    ok &= mbar_wait(bar_kv + (st ^ 1), ((kv_count + 1) >> 1) & 1);
+                    tc_fence_after();
+                    issue_scores(tmem + (st ^ 1) * 128, sK + (st ^ 1) * kTileBytes);
+                }
             }
             ok &= mbar_wait(bar_o, ph);
             tc_fence_after();
