@@ -65,10 +65,10 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
         part += __shfl_xor_sync(0xffffffffu, part, 1);
         part += __shfl_xor_sync(0xffffffffu, part, 2);
         part += __shfl_xor_sync(0xffffffffu, part, 4);
-        if (dc == 0) P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + i] = part;
+        if (P.delta && dc == 0) P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + i] = part;
         const size_t dst = (static_cast<size_t>(b) * P.Ncap + i) * chunks_row + c;
         if (P.dog) P.dog[dst] = vd;
-        if (n_sel > kTile) {                          // a single key tile writes dq directly, nothing to accumulate
+        if (P.dq_acc && n_sel > kTile) {              // a single key tile writes dq directly, nothing to accumulate
             P.dq_acc[2 * dst] = make_float4(0.f, 0.f, 0.f, 0.f);
             P.dq_acc[2 * dst + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
@@ -80,7 +80,10 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
 // ---------------------------------------------------------------------------------------------------------
 struct BwdParams {
     const float* lse;       // [B, H, N]
-    const float* delta;     // [B, H, Ncap]
+    const __nv_bfloat16* o; // [B, N, H, D] forward output (rows 0 .. n_sel-1), for Delta
+    const float* delta;     // [B, H, Ncap] precomputed Delta, or NULL: computed here from o and dO
+    TileSource src;         // where Q, K, V tiles come from
+    TileSource src_do;      // where dO tiles come from
     float* dq_acc;          // [B, Ncap, H, 64]
     __nv_bfloat16* dq;      // [B, N, H, D]; written here only when there is a single key tile
     __nv_bfloat16* dk;
@@ -132,7 +135,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint64_t* bar_s = bars + 3;
     uint64_t* bar_g = bars + 4;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-    float* s_stat = reinterpret_cast<float*>(smem_dyn + 64);      // [2 stages][lse (log2 domain) 128 | Delta 128]
+    float* s_stat = reinterpret_cast<float*>(smem_dyn + 64);      // [2 stages][128] lse of the query tile, log2 domain
+    float* s_dpart = s_stat + 2 * kTile;                          // [2 halves][128] partial Delta = sum over 32 head dims of dO O
     unsigned char* sK = align_tiles(smem_dyn + 64 + 4 * kTile * sizeof(float));
     unsigned char* sV = sK + kTileBytes;
     unsigned char* sQ = sV + kTileBytes;            // 2 stages
@@ -195,40 +199,65 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         tc_commit(bar_s);
     };
 
-    // row statistic of query `qrow`: threads 0..127 fetch lse (log2 domain), threads 128..255 fetch Delta
-    auto load_stat = [&](int b, int h, int qrow) -> float {
-        if (qrow >= n_sel) return half == 0 ? INFINITY : 0.f;
-        return half == 0 ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f
-                         : P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow];
+    // lse of query `qrow` in the log2 domain (fetched by the threads of half 0; +inf switches a missing query off)
+    auto load_lse = [&](int b, int h, int qrow) -> float {
+        if (half != 0) return 0.f;
+        return qrow < n_sel ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
+    };
+    // this thread's 32 head dimensions (64 bytes) of forward-output row `qrow`, zeros when there is no such row
+    auto load_o = [&](int b, int h, int qrow, uint4* dst) {
+        const bool have = qrow < n_sel && half * 32 < P.D;
+        const uint4* src = reinterpret_cast<const uint4*>(P.o + ((static_cast<size_t>(b) * P.N + (have ? qrow : 0)) * P.H + h) * P.D + (have ? half * 32 : 0));
+#pragma unroll
+        for (int x = 0; x < 4; ++x) dst[x] = have ? __ldg(src + x) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    // precomputed Delta of query `qrow` (fetched by the threads of half 1)
+    auto load_delta = [&](int b, int h, int qrow) -> float {
+        if (half != 1 || !P.delta) return 0.f;
+        return qrow < n_sel ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
+    };
+    auto dot8 = [](uint4 a, uint4 g) -> float {
+        const float2 a0 = unpack2(a.x), a1 = unpack2(a.y), a2 = unpack2(a.z), a3 = unpack2(a.w);
+        const float2 g0 = unpack2(g.x), g1 = unpack2(g.y), g2 = unpack2(g.z), g3 = unpack2(g.w);
+        return a0.x * g0.x + a0.y * g0.y + a1.x * g1.x + a1.y * g1.y + a2.x * g2.x + a2.y * g2.y + a3.x * g3.x + a3.y * g3.y;
     };
 
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
         const int jt = item % n_q;
         const int h = (item / n_q) % P.H;
         const int b = item / (n_q * P.H);
-        if (tid == 0) {             // every MMA of the previous item has completed: K, V and both Q/dO stages are free
-            mbar_expect_tx(bar_kv, 2 * kTileBytes);
-            tma_load_4d(sK, &map_k, bar_kv, 0, h, jt * kTile, b);
-            tma_load_4d(sV, &map_v, bar_kv, 0, h, jt * kTile, b);
+        if (warp == 0) {            // every MMA of the previous item has completed: K, V and both Q/dO stages are free
             const uint32_t st0 = q_count & 1;
-            mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
-            tma_load_4d(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, 0, h, 0, b);
-            tma_load_4d(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, 0, h, 0, b);
+            if (tid == 0) {
+                mbar_expect_tx(bar_kv, 2 * kTileBytes);
+                mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
+            }
+            __syncwarp();
+            load_tile(sK, &map_k, bar_kv, P.src, jt * kTile, n_sel, h, b, P.H);
+            load_tile(sV, &map_v, bar_kv, P.src, jt * kTile, n_sel, h, b, P.H);
+            load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, P.src, 0, n_sel, h, b, P.H);
+            load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, P.src_do, 0, n_sel, h, b, P.H);
         }
-        s_stat[(q_count & 1) * 2 * kTile + tid] = load_stat(b, h, row);
+        if (half == 0) s_stat[(q_count & 1) * kTile + row] = load_lse(b, h, row);
+        uint4 o_cur[4], o_next[4];
+        float dl_cur = load_delta(b, h, row), dl_next = 0.f;
+        if (!P.delta) load_o(b, h, row, o_cur);
         const int key = jt * kTile + row;               // this thread's key row
         const bool key_valid = key < n_sel;
 
         for (int i = 0; i < n_q; ++i, ++q_count) {
             const uint32_t st = q_count & 1, ph = q_count & 1;
-            float next_stat = 0.f;
+            float next_lse = 0.f;
             if (i + 1 < n_q) {
-                if (tid == 0) {                          // the other stage was released by the wait on bar_g of the previous tile
-                    mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);
-                    tma_load_4d(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), 0, h, (i + 1) * kTile, b);
-                    tma_load_4d(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), 0, h, (i + 1) * kTile, b);
+                if (warp == 0) {                         // the other stage was released by the wait on bar_g of the previous tile
+                    if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);
+                    __syncwarp();
+                    load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), P.src, (i + 1) * kTile, n_sel, h, b, P.H);
+                    load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), P.src_do, (i + 1) * kTile, n_sel, h, b, P.H);
                 }
-                next_stat = load_stat(b, h, (i + 1) * kTile + row);      // lands while this tile is processed
+                next_lse = load_lse(b, h, (i + 1) * kTile + row);        // both land while this tile is processed
+                dl_next = load_delta(b, h, (i + 1) * kTile + row);
+                if (!P.delta) load_o(b, h, (i + 1) * kTile + row, o_next);
             }
             if (tid == 0 && i == 0) {                    // later tiles: issued right behind the previous tile's products
                 ok &= mbar_wait(bar_kv, n_done & 1);
@@ -236,13 +265,24 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tc_fence_after();
                 issue_scores(sQ + st * kTileBytes, sdO + st * kTileBytes);
             }
+            if (P.delta) {
+                s_dpart[half * kTile + row] = dl_cur;    // half 1 holds the value, half 0 contributes zero
+            } else {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
+                ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
+                const unsigned char* do_row = sdO + st * kTileBytes + row * kRowBytes;
+                float part = 0.f;
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+                    part += dot8(o_cur[x], *reinterpret_cast<const uint4*>(do_row + (((half * 4 + x) ^ (row & 7)) << 4)));
+                s_dpart[half * kTile + row] = part;
+            }
             __syncthreads();                             // row statistics of this stage visible
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
 
             // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
-            const float* lse2 = s_stat + st * 2 * kTile + half * 64;
-            const float* dlt = lse2 + kTile;
+            const float* lse2 = s_stat + st * kTile + half * 64;
+            const float* dlt = s_dpart + half * 64;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 float sv[32], dp[32];
@@ -252,7 +292,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 #pragma unroll
                 for (int x = 0; x < 32; x += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 32 + x);
-                    const float4 d4 = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
+                    const float4 da = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
+                    const float4 db = *reinterpret_cast<const float4*>(dlt + kTile + c * 32 + x);
+                    const float4 d4 = make_float4(da.x + db.x, da.y + db.y, da.z + db.z, da.w + db.w);
                     const float p0 = fast_exp2(fmaf(sv[x + 0], P.scale_log2, -l4.x)), p1 = fast_exp2(fmaf(sv[x + 1], P.scale_log2, -l4.y));
                     const float p2 = fast_exp2(fmaf(sv[x + 2], P.scale_log2, -l4.z)), p3 = fast_exp2(fmaf(sv[x + 3], P.scale_log2, -l4.w));
                     sv[x + 0] = p0; sv[x + 1] = p1; sv[x + 2] = p2; sv[x + 3] = p3;
@@ -292,7 +334,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     issue_scores(sQ + (st ^ 1) * kTileBytes, sdO + (st ^ 1) * kTileBytes);
                 }
             }
-            if (i + 1 < n_q) s_stat[(st ^ 1) * 2 * kTile + tid] = next_stat;      // read only after the next top-of-loop barrier
+            if (i + 1 < n_q) {
+                if (half == 0) s_stat[(st ^ 1) * kTile + row] = next_lse;        // read only after the next top-of-loop barrier
+                dl_cur = dl_next;
+                if (!P.delta) {
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) o_cur[x] = o_next[x];
+                }
+            }
             ok &= mbar_wait(bar_g, ph);
             tc_fence_after();
             {   // dQ_i: tensor-memory lane = query row; this thread drains 32 of the 64 head-dimension columns
@@ -404,14 +453,19 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     const bool staged = attn_uses_staging(c, sel_idx);
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
 
-    PrepParams R{};
-    R.o = static_cast<const uint4*>(o); R.d_o = static_cast<const uint4*>(d_o);
-    R.dog = staged ? reinterpret_cast<uint4*>(base + w.dog) : nullptr;
-    R.delta = reinterpret_cast<float*>(base + w.delta);
-    R.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
-    R.n_sel = sel_idx ? n_sel : nullptr;
-    R.N = c.N; R.Ncap = w.Ncap; R.H = c.H; R.D = c.D;
-    {
+    const bool gathered = attn_uses_gather(c, sel_idx);
+    // Delta is precomputed when the number of tokens is known here (no selection) and there is more than one key tile:
+    // every key-tile CTA would otherwise recompute it.  With a selection the count lives on the device and the main
+    // kernel computes Delta itself.
+    const bool pre_delta = sel_idx == nullptr && c.N > kTile;
+    if (staged || pre_delta) {       // D = 32 also needs a zero-padded copy of dO next to the staged Q', K', V'
+        PrepParams R{};
+        R.o = static_cast<const uint4*>(o); R.d_o = static_cast<const uint4*>(d_o);
+        R.dog = staged ? reinterpret_cast<uint4*>(base + w.dog) : nullptr;
+        R.delta = pre_delta ? reinterpret_cast<float*>(base + w.delta) : nullptr;
+        R.dq_acc = nullptr;
+        R.n_sel = sel_idx ? n_sel : nullptr;
+        R.N = c.N; R.Ncap = w.Ncap; R.H = c.H; R.D = c.D;
         const long long work = static_cast<long long>(w.Ncap) * c.H * 8;
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 4 * sm_count() / c.B);              // about four CTAs per SM in total
@@ -426,6 +480,12 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mdo, base + w.dog, c.B, w.Ncap, w.Ncap, c.H)) return st;
+    } else if (gathered) {
+        const long long rows = static_cast<long long>(c.B) * c.N * c.H;
+        if (int st = make_row_map(&mq, q, rows)) return st;
+        if (int st = make_row_map(&mk, k, rows)) return st;
+        if (int st = make_row_map(&mv, v, rows)) return st;
+        if (int st = make_row_map(&mdo, d_o, rows)) return st;
     } else {
         if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
         if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
@@ -433,7 +493,11 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         if (int st = make_tile_map(&mdo, d_o, c.B, c.N, c.N, c.H)) return st;
     }
     BwdParams P{};
-    P.lse = lse; P.delta = R.delta; P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
+    P.lse = lse; P.o = static_cast<const __nv_bfloat16*>(o); P.delta = pre_delta ? reinterpret_cast<const float*>(base + w.delta) : nullptr;
+    P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
+    P.src.idx = sel_idx; P.src.gathered = gathered ? 1 : 0; P.src.tokens = c.N; P.src.rows_total = c.B * c.N * c.H;
+    P.src_do = P.src;
+    P.src_do.idx = nullptr;         // dO rows are already compact: slot j is row j
     P.dq = static_cast<__nv_bfloat16*>(dq); P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
     P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);

@@ -39,6 +39,10 @@ inline AttnWs attn_layout(const vardrop_attn_cfg& c) {
 // Tensor map over a [B, tokens, H, 64] bf16 tensor: box = one (b, h) tile of 128 tokens x 64 elements,
 // 128-byte swizzle, out-of-range rows read as zero.  `tokens` is the extent the copy engine may touch,
 // `token_stride` the allocated tokens per instance.
+// Tensor map over the same memory seen as [rows, 64] bf16 (rows = B * tokens * H) for row gathers: box = one row,
+// 128-byte swizzle, rows outside the tensor read as zero.
+int make_row_map(CUtensorMap* map, const void* base, long long rows);
+
 // Number of SMs of the current device (cached per thread and device).
 int sm_count();
 
@@ -49,8 +53,39 @@ __device__ __forceinline__ unsigned char* align_tiles(unsigned char* p) {
     return reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~static_cast<uintptr_t>(1023));
 }
 
+// How a 128-token operand tile reaches shared memory.
+//   tiled    one 4-D box of the [B, tokens, H, 64] tensor (tokens tok0 .. tok0 + 127 of head h, instance b)
+//   gathered 32 row gathers of 4 rows each from the [rows, 64] view: slot j of the tile is variate idx[tok0 + j]
+//            (idx = NULL: the slot itself) while tok0 + j < n_valid, and a row past the end (zeros) otherwise.
+// Called by all 32 lanes of one warp; `lane0_expect` bytes are announced on the barrier by lane 0 first.
+struct TileSource {
+    const int32_t* idx;    // gather indices (NULL: identity)
+    int gathered;          // 0: tiled box, 1: row gathers
+    int tokens;            // tokens per instance in the gathered tensor
+    int rows_total;        // B * tokens * H
+};
+__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* map, uint64_t* bar, const TileSource& src, int tok0, int n_valid,
+                                          int h, int b, int H) {
+    const int lane = threadIdx.x & 31;
+    if (!src.gathered) {
+        if (lane == 0) tma_load_4d(dst, map, bar, 0, h, tok0, b);
+        return;
+    }
+    int rows[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int slot = tok0 + 4 * lane + e;
+        int n = -1;
+        if (slot < n_valid) n = src.idx ? src.idx[slot] : slot;
+        rows[e] = n >= 0 ? (b * src.tokens + n) * H + h : src.rows_total;
+    }
+    tma_gather4(dst + lane * 4 * kRowBytes, map, bar, 0, rows[0], rows[1], rows[2], rows[3]);
+}
+
 // Operands either come straight from the caller's tensors (all-token path at D = 64) or from the staged
-// copies in the workspace (a selection is given, or D = 32 needs padding).
-inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return sel_idx != nullptr || c.D != kDP; }
+// copies in the workspace (D = 32 needs padding to 64).
+inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t*) { return c.D != kDP; }
+// With D = 64 and a selection, the kept rows are gathered by the copy engine straight from the caller's tensors.
+inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D == kDP && sel_idx != nullptr; }
 
 }  // namespace vardrop

@@ -56,10 +56,25 @@ int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int tok
     return VARDROP_OK;
 }
 
+int make_row_map(CUtensorMap* map, const void* base, long long rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(kDP), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(kRowBytes)};
+    const cuuint32_t box[2] = {kDP, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled (row view) failed with code %d", static_cast<int>(r));
+    return VARDROP_OK;
+}
+
 int attn_validate(const vardrop_attn_cfg& c) {
     if (c.B < 1 || c.N < 1 || c.H < 1) return fail(VARDROP_ERR_INVALID_ARG, "attention: B, N, H >= 1 required (B=%d N=%d H=%d)", c.B, c.N, c.H);
     if (c.D != 32 && c.D != 64) return fail(VARDROP_ERR_UNSUPPORTED, "attention: head dimension %d (32 or 64 supported)", c.D);
     if (c.N > 65536) return fail(VARDROP_ERR_UNSUPPORTED, "attention: N=%d above 65536", c.N);
+    if (static_cast<long long>(c.B) * c.N * c.H >= (1ll << 31)) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B*N*H above 2^31");
     if (c.H > 65535 || c.B > 65535) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B or H above 65535");
     if (!(c.sm_scale >= 0.f)) return fail(VARDROP_ERR_INVALID_ARG, "attention: sm_scale must be >= 0 (0 selects 1/sqrt(D))");
     return VARDROP_OK;
@@ -108,7 +123,9 @@ struct FwdParams {
     float* lse;
     const int32_t* n_sel;   // NULL: all N tokens
     int* status;
-    int B, N, H, D;
+    float4* dq_acc;         // [B, Ncap, H, 64] fp32: zeroed here for the backward pass when it will accumulate into it
+    TileSource src;         // where Q, K, V tiles come from
+    int B, N, Ncap, H, D;
     float scale_log2;       // sm_scale * log2(e)
 };
 
@@ -208,13 +225,23 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
         const int qt = item % n_kv;
         const int h = (item / n_kv) % P.H;
         const int b = item / (n_kv * P.H);
-        if (tid == 0) {             // every MMA of the previous item has completed: Q and both ring stages are free
-            mbar_expect_tx(bar_q, kTileBytes);
-            tma_load_4d(sQ, &map_q, bar_q, 0, h, qt * kTile, b);
+        if (warp == 0) {            // every MMA of the previous item has completed: Q and both ring stages are free
             const uint32_t st0 = kv_count & 1;
-            mbar_expect_tx(bar_kv + st0, 2 * kTileBytes);
-            tma_load_4d(sK + st0 * kTileBytes, &map_k, bar_kv + st0, 0, h, 0, b);
-            tma_load_4d(sV + st0 * kTileBytes, &map_v, bar_kv + st0, 0, h, 0, b);
+            if (tid == 0) {
+                mbar_expect_tx(bar_q, kTileBytes);
+                mbar_expect_tx(bar_kv + st0, 2 * kTileBytes);
+            }
+            __syncwarp();
+            load_tile(sQ, &map_q, bar_q, P.src, qt * kTile, n_sel, h, b, P.H);
+            load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, P.src, 0, n_sel, h, b, P.H);
+            load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, P.src, 0, n_sel, h, b, P.H);
+        }
+        if (n_kv > 1) {             // the backward pass will add per-key-tile pieces of dQ' into the accumulator: clear this tile's rows
+#pragma unroll
+            for (int x = 0; x < kDP / 4; ++x) {          // 16 consecutive threads clear one 256-byte row
+                const int idx = x * kFwdThreads + tid, r = idx >> 4, c4 = idx & 15;
+                P.dq_acc[((static_cast<size_t>(b) * P.Ncap + qt * kTile + r) * P.H + h) * (kDP / 4) + c4] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
 
         float o_acc[kDP];
@@ -225,12 +252,13 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
         for (int j = 0; j < n_kv; ++j, ++kv_count) {
             const uint32_t st = kv_count & 1;
             const uint32_t ph = kv_count & 1;            // bar_s / bar_o complete once per key tile
+            if (warp == 0 && j + 1 < n_kv) {             // the other stage was released by the wait on bar_o of the previous tile
+                if (tid == 0) mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
+                __syncwarp();
+                load_tile(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), P.src, (j + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), P.src, (j + 1) * kTile, n_sel, h, b, P.H);
+            }
             if (tid == 0) {
-                if (j + 1 < n_kv) {                      // the other stage was released by the wait on bar_o of the previous tile
-                    mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
-                    tma_load_4d(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
-                    tma_load_4d(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), 0, h, (j + 1) * kTile, b);
-                }
                 if (j == 0) {                            // later tiles: issued right behind the previous tile's P V
                     ok &= mbar_wait(bar_q, n_done & 1);
                     ok &= mbar_wait(bar_kv + st, (kv_count >> 1) & 1);
@@ -355,6 +383,11 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+    } else if (attn_uses_gather(c, sel_idx)) {
+        const long long rows = static_cast<long long>(c.B) * c.N * c.H;
+        if (int st = make_row_map(&mq, q, rows)) return st;
+        if (int st = make_row_map(&mk, k, rows)) return st;
+        if (int st = make_row_map(&mv, v, rows)) return st;
     } else {
         if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
         if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
@@ -363,7 +396,10 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
     FwdParams P{};
     P.o = static_cast<__nv_bfloat16*>(o); P.lse = lse; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);
-    P.B = c.B; P.N = c.N; P.H = c.H; P.D = c.D;
+    P.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
+    P.src.idx = sel_idx; P.src.gathered = attn_uses_gather(c, sel_idx) ? 1 : 0; P.src.tokens = c.N;
+    P.src.rows_total = c.B * c.N * c.H;
+    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
     P.scale_log2 = scale * 1.4426950408889634f;
     static thread_local int attr_dev = -1;
