@@ -142,6 +142,36 @@ __device__ __forceinline__ void fft_stage(const float2* __restrict__ in, float2*
     }
 }
 
+// First Stockham stage (Ns = 1: no twiddles, butterfly j writes out[j R + r]) reading the windows straight from global
+// memory: transform p carries window 2p of the pass in its real part and window 2p + 1 (if any) in its imaginary part.
+template <int R>
+__device__ __forceinline__ void fft_first_stage(const HashParams& P, float2* __restrict__ out, int n_win, int row0, int b0, int cw,
+                                                FastDiv div_lr) {
+    const uint32_t L = P.L, LR = div_lr.d;
+    const uint32_t n_fft = (n_win + 1) >> 1;
+    const uint32_t total = n_fft * LR;
+    for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+        const uint32_t p = fd_div(t, div_lr);
+        const uint32_t j = t - p * LR;
+        const float* src[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const uint32_t wl = 2 * p + e;
+            const uint32_t r = cw == P.chunk ? fd_div(wl, P.div_chunk) : wl / static_cast<uint32_t>(cw);
+            const uint32_t bi = wl - r * cw;
+            const size_t w = P.scope == 0 ? static_cast<size_t>(b0 + bi) * P.N + (row0 + r) : static_cast<size_t>(row0 + r);
+            src[e] = wl < static_cast<uint32_t>(n_win) ? P.x + w * L + j : nullptr;
+        }
+        float2 v[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) v[r] = make_float2(__ldg(src[0] + r * LR), src[1] ? __ldg(src[1] + r * LR) : 0.f);
+        small_dft<R>(v);
+        float2* dst = out + p * L + j * R;
+#pragma unroll
+        for (int r = 0; r < R; ++r) dst[r] = v[r];
+    }
+}
+
 __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int L = P.L, nf = P.nf;
@@ -152,10 +182,11 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
     float2* buf1 = buf0 + static_cast<size_t>(max_fft) * L;
     float* acc = reinterpret_cast<float*>(buf1 + static_cast<size_t>(max_fft) * L);   // [rows_per_cta, nf]
 
-    for (int m = threadIdx.x; m < L; m += blockDim.x) {
-        double s, c;
-        sincospi(2.0 * static_cast<double>(m) / static_cast<double>(L), &s, &c);
-        tw[m] = make_float2(static_cast<float>(c), static_cast<float>(-s));
+    for (int m = threadIdx.x; m < L; m += blockDim.x) {      // w^m = exp(-2 pi i m / L); the angle is folded to |m'| <= L / 2 first
+        const int mf = 2 * m > L ? m - L : m;
+        float s, c;
+        sincospif(2.f * static_cast<float>(mf) / static_cast<float>(L), &s, &c);
+        tw[m] = make_float2(c, -s);
     }
     const int row0 = blockIdx.x * P.rows_per_cta;
     const int rows = min(P.rows_per_cta, P.rows_total - row0);
@@ -166,42 +197,18 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
         const int n_win = rows * cw;
         const int n_fft = (n_win + 1) / 2;
         __syncthreads();
-        // ---- load: window wl = r * cw + bi of the pass -> component (wl & 1) of transform wl >> 1 -------
-        {
-            float* dstf = reinterpret_cast<float*>(buf0);
-            if ((L & 3) == 0) {
-                const uint32_t L4 = L >> 2;
-                for (uint32_t idx = threadIdx.x; idx < static_cast<uint32_t>(n_win) * L4; idx += blockDim.x) {
-                    const uint32_t wl = fd_div(idx, P.div_L4);
-                    const uint32_t t4 = idx - wl * L4;
-                    const uint32_t r = cw == P.chunk ? fd_div(wl, P.div_chunk) : wl / static_cast<uint32_t>(cw);
-                    const uint32_t bi = wl - r * cw;
-                    const int row = row0 + r;
-                    const size_t w = P.scope == 0 ? static_cast<size_t>(b0 + bi) * P.N + row : static_cast<size_t>(row);
-                    const float4 val = __ldg(reinterpret_cast<const float4*>(P.x + w * L) + t4);
-                    float* d = dstf + (static_cast<size_t>(wl >> 1) * L + t4 * 4) * 2 + (wl & 1);
-                    d[0] = val.x; d[2] = val.y; d[4] = val.z; d[6] = val.w;
-                }
-            } else {
-                for (uint32_t idx = threadIdx.x; idx < static_cast<uint32_t>(n_win) * L; idx += blockDim.x) {
-                    const uint32_t wl = fd_div(idx, P.div_L);
-                    const uint32_t t = idx - wl * L;
-                    const uint32_t r = cw == P.chunk ? fd_div(wl, P.div_chunk) : wl / static_cast<uint32_t>(cw);
-                    const uint32_t bi = wl - r * cw;
-                    const int row = row0 + r;
-                    const size_t w = P.scope == 0 ? static_cast<size_t>(b0 + bi) * P.N + row : static_cast<size_t>(row);
-                    dstf[(static_cast<size_t>(wl >> 1) * L + t) * 2 + (wl & 1)] = __ldg(P.x + w * L + t);
-                }
-            }
-            if (n_win & 1) {                                 // last transform has no second window
-                for (int t = threadIdx.x; t < L; t += blockDim.x) dstf[(static_cast<size_t>(n_fft - 1) * L + t) * 2 + 1] = 0.f;
-            }
-        }
-        __syncthreads();
-        // ---- mixed-radix Stockham FFT, ping-pong between the two buffers -------------------------------
+        // ---- mixed-radix Stockham FFT, ping-pong between the two buffers; the first stage reads global memory --
         float2* cur = buf0;
         float2* oth = buf1;
-        for (int s = 0; s < P.n_stages; ++s) {
+        switch (P.radix[0]) {
+            case 2: fft_first_stage<2>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            case 3: fft_first_stage<3>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            case 4: fft_first_stage<4>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            case 5: fft_first_stage<5>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            default: fft_first_stage<7>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+        }
+        __syncthreads();
+        for (int s = 1; s < P.n_stages; ++s) {
             switch (P.radix[s]) {
                 case 2: fft_stage<2>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
                 case 3: fft_stage<3>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
@@ -236,38 +243,37 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
     }
     __syncthreads();
 
-    // ---- mean, top-k ranking (descending amplitude, lower bin first on ties), packing ---------------------
+    // ---- top-k ranking (descending amplitude, lower bin first on ties), packing ------------------------------
+    // Ranking the batch sums ranks the means.  A candidate is coded as (amplitude bits, ~bin): amplitudes are
+    // non-negative, so unsigned comparison of the code orders by amplitude and then by lower bin.
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
-    const float n_avg = static_cast<float>(P.win_per_row);
+    const float inv_n = 1.f / static_cast<float>(P.win_per_row);
     for (int r = warp; r < rows; r += n_warps) {
         float* a = acc + r * nf;
         const int row = row0 + r;
         bool bad = false;
         for (int fi = lane; fi < nf; fi += 32) {
-            const float mean = a[fi] / n_avg;
-            a[fi] = mean;
-            bad |= !isfinite(mean);
-            if (P.amp_dbg) P.amp_dbg[static_cast<size_t>(row) * nf + fi] = mean;
+            const float sum = a[fi];
+            bad |= !isfinite(sum);
+            if (P.amp_dbg) P.amp_dbg[static_cast<size_t>(row) * nf + fi] = sum * inv_n;
         }
         if (__any_sync(0xffffffffu, bad) && lane == 0) set_status(P.status, VARDROP_ERR_NONFINITE);
-        __syncwarp();
         uint64_t key = 0;
         for (int rank = 0; rank < P.k; ++rank) {
-            float best = -2.f;
-            int best_f = 0x7fffffff;
+            uint64_t best = 0;                               // code 0 = nothing found (taken entries are negative)
             for (int fi = lane; fi < nf; fi += 32) {
                 const float val = a[fi];
-                if (val > best) { best = val; best_f = fi; }
+                const uint64_t code = (static_cast<uint64_t>(__float_as_uint(val)) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(fi));
+                if (val >= 0.f && code > best) best = code;
             }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-                const int of = __shfl_xor_sync(0xffffffffu, best_f, off);
-                if (ov > best || (ov == best && of < best_f)) { best = ov; best_f = of; }
+                const uint64_t other = __shfl_xor_sync(0xffffffffu, best, off);
+                best = other > best ? other : best;
             }
-            if (best_f == 0x7fffffff) best_f = 0;            // only reachable with non-finite input (status is set)
+            const int best_f = best ? static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(best)) : 0;      // 0 only with non-finite input
             if (lane == 0) {
-                a[best_f] = -1.f;                            // amplitudes are >= 0: -1 removes the winner
+                a[best_f] = -1.f;                            // removes the winner
                 if (P.freqs) P.freqs[static_cast<size_t>(row) * P.k + rank] = P.f_lo + best_f;
             }
             key = (key << 12) | static_cast<uint64_t>(P.f_lo + best_f);
