@@ -191,6 +191,24 @@ def time_region(torch, fn, steps, dist_barrier):
     return start.elapsed_time(stop)
 
 
+def recorded_traffic(kernel, workload):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when there is no capture for this
+    workload or the kernel's source file has changed since the capture."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as fh:
+        rec = json.load(fh).get(kernel)
+    if not rec or rec.get("workload") != workload:
+        return None
+    src = os.path.join(ROOT, "paper_2501_14183_b200", "csrc", rec["source_file"])
+    with open(src, "rb") as fh:
+        if hashlib.sha256(fh.read()).hexdigest() != rec["source_sha256"]:
+            return None
+    return rec["dram_bytes_per_launch"]
+
+
 def kernel_work(w, n_sel):
     """Algorithmic bytes / flops of one launch of each kernel (what the method must move or compute)."""
     row = w.H * w.D * 2
@@ -308,7 +326,7 @@ def run_gpu(args):
     kernels = kernel_table(per_kernel, kernel_work(w, n_sel), peaks)
     top = max(kernels, key=lambda k: kernels[k]["share"])
     roofline = {"kernel": top, "bound": kernels[top]["bound"], "achieved": kernels[top]["achieved"], "peak": kernels[top]["peak"],
-                "unit": kernels[top]["unit"], "frac": kernels[top]["frac"], "traffic": None,
+                "unit": kernels[top]["unit"], "frac": kernels[top]["frac"], "traffic": recorded_traffic(top, w.name),
                 "peak_source": f"{peak_kind} (burst figure for tensor work)",
                 "timing": "CUDA events around every launch, second pass of the same K steps",
                 "ms_per_step_with_timer_armed": ms_armed / args.steps}

@@ -44,6 +44,7 @@ struct PrepParams {
 // one thread per 16-byte chunk of a staged (token, head) row; the 8 threads of a row reduce Delta by shuffles
 __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
     const int n_sel = P.n_sel ? *P.n_sel : P.N;
+    if (!P.dog && n_sel <= kTile) return;            // a single key tile: the main kernel computes Delta itself
     const int n_fill = min(P.Ncap, (n_sel + kTile - 1) / kTile * kTile);
     const int b = blockIdx.y;
     const int chunks_row = P.H * 8;
@@ -186,6 +187,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint32_t q_count = 0;       // query tiles consumed so far by this CTA: stage = q_count & 1
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
     const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
+    const bool use_delta = P.delta != nullptr && n_q > 1;      // precomputed Delta exists only when there are several key tiles
 
     // S^T = K Q^T and dP^T = V dO^T of one query tile (issued by one thread), completion on bar_s
     auto issue_scores = [&](const unsigned char* q_tile, const unsigned char* do_tile) {
@@ -213,7 +215,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     };
     // precomputed Delta of query `qrow` (fetched by the threads of half 1)
     auto load_delta = [&](int b, int h, int qrow) -> float {
-        if (half != 1 || !P.delta) return 0.f;
+        if (half != 1 || !use_delta) return 0.f;
         return qrow < n_sel ? P.delta[(static_cast<size_t>(b) * P.H + h) * P.Ncap + qrow] : 0.f;
     };
     auto dot8 = [](uint4 a, uint4 g) -> float {
@@ -241,7 +243,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         if (half == 0) s_stat[(q_count & 1) * kTile + row] = load_lse(b, h, row);
         uint4 o_cur[4], o_next[4];
         float dl_cur = load_delta(b, h, row), dl_next = 0.f;
-        if (!P.delta) load_o(b, h, row, o_cur);
+        if (!use_delta) load_o(b, h, row, o_cur);
         const int key = jt * kTile + row;               // this thread's key row
         const bool key_valid = key < n_sel;
 
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
                 next_lse = load_lse(b, h, (i + 1) * kTile + row);        // both land while this tile is processed
                 dl_next = load_delta(b, h, (i + 1) * kTile + row);
-                if (!P.delta) load_o(b, h, (i + 1) * kTile + row, o_next);
+                if (!use_delta) load_o(b, h, (i + 1) * kTile + row, o_next);
             }
             if (tid == 0 && i == 0) {                    // later tiles: issued right behind the previous tile's products
                 ok &= mbar_wait(bar_kv, n_done & 1);
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tc_fence_after();
                 issue_scores(sQ + st * kTileBytes, sdO + st * kTileBytes);
             }
-            if (P.delta) {
+            if (use_delta) {
                 s_dpart[half * kTile + row] = dl_cur;    // half 1 holds the value, half 0 contributes zero
             } else {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
                 ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
@@ -337,7 +339,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (i + 1 < n_q) {
                 if (half == 0) s_stat[(st ^ 1) * kTile + row] = next_lse;        // read only after the next top-of-loop barrier
                 dl_cur = dl_next;
-                if (!P.delta) {
+                if (!use_delta) {
 #pragma unroll
                     for (int x = 0; x < 4; ++x) o_cur[x] = o_next[x];
                 }
@@ -454,10 +456,10 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
 
     const bool gathered = attn_uses_gather(c, sel_idx);
-    // Delta is precomputed when the number of tokens is known here (no selection) and there is more than one key tile:
-    // every key-tile CTA would otherwise recompute it.  With a selection the count lives on the device and the main
-    // kernel computes Delta itself.
-    const bool pre_delta = sel_idx == nullptr && c.N > kTile;
+    // Delta is precomputed by a small kernel when there can be many key tiles (every key-tile CTA would otherwise
+    // recompute it): without a selection, and on the staged path, where that kernel runs anyway to stage dO.  On the
+    // gathered path (few tiles) the main kernel computes Delta itself.
+    const bool pre_delta = sel_idx == nullptr ? c.N > kTile : staged;
     if (staged || pre_delta) {       // D = 32 also needs a zero-padded copy of dO next to the staged Q', K', V'
         PrepParams R{};
         R.o = static_cast<const uint4*>(o); R.d_o = static_cast<const uint4*>(d_o);

@@ -82,10 +82,15 @@ __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap*
     tma_gather4(dst + lane * 4 * kRowBytes, map, bar, 0, rows[0], rows[1], rows[2], rows[3]);
 }
 
-// Operands either come straight from the caller's tensors (all-token path at D = 64) or from the staged
-// copies in the workspace (D = 32 needs padding to 64).
-inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t*) { return c.D != kDP; }
-// With D = 64 and a selection, the kept rows are gathered by the copy engine straight from the caller's tensors.
-inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D == kDP && sel_idx != nullptr; }
+// Three ways for the operand tiles to reach shared memory:
+//   direct   4-D boxes of the caller's tensors                       (no selection, D = 64)
+//   gathered row gathers of the kept variates from the caller's tensors   (selection, D = 64, N <= kGatherMaxN: the kept set
+//            is at most a few tiles, so re-gathering rows per tile pair costs less than a staging pass)
+//   staged   4-D boxes of compacted copies in the workspace, written by the gather kernel   (D = 32, which is also
+//            zero-padded to 64 there; or a selection at large N, where every tile is re-read many times and
+//            contiguous, L2-resident tiles pay for the extra pass)
+constexpr int kGatherMaxN = 512;
+inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D != kDP || (sel_idx != nullptr && c.N > kGatherMaxN); }
+inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D == kDP && sel_idx != nullptr && c.N <= kGatherMaxN; }
 
 }  // namespace vardrop
