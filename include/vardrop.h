@@ -174,8 +174,9 @@ int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, i
  * n_sel       [1] int32 on the device, number of valid entries of sel_idx; ignored when sel_idx is NULL.
  * o           [B, N, H, D] bf16 out; rows 0..n_sel-1 of every instance hold O', the rest is untouched.
  * lse         [B, H, N] float32 out; entries 0..n_sel-1 valid.
- * ws          scratch of vardrop_attn_workspace_bytes.  After the call it holds the gathered Q', K', V';
- *             vardrop_attn_bwd for the same step must be given the same, unmodified workspace.
+ * ws          scratch of vardrop_attn_workspace_bytes.  After the call it holds what the backward pass of the same
+ *             step needs (staged Q', K', V' where the library stages them, a cleared dQ' accumulator):
+ *             vardrop_attn_bwd must be given the same, unmodified workspace, once per forward call.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     int32_t B, N, H, D;
