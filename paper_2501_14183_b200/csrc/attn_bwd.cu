@@ -99,7 +99,7 @@ struct BwdParams {
 constexpr int kBwdThreads = 256;       // two threads per tensor-memory lane: each takes one 64-column half
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 4 * kTileBytes /*Q, dO x 2 stages*/ +
-                              4 * kTileBytes /*P^T, dS^T*/;
+                              4 * kTileBytes /*P^T, dS^T*/ + 2 * kTileBytes /*dQ tile, fp32, two 32-column halves*/;
 
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
@@ -123,7 +123,8 @@ __device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                    const __grid_constant__ CUtensorMap map_k,
                                                                    const __grid_constant__ CUtensorMap map_v,
-                                                                   const __grid_constant__ CUtensorMap map_do, const BwdParams P) {
+                                                                   const __grid_constant__ CUtensorMap map_do,
+                                                                   const __grid_constant__ CUtensorMap map_acc, const BwdParams P) {
     const int n_sel = P.n_sel ? *P.n_sel : P.N;
     const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles
     const int n_items = n_q * P.H * P.B;                       // work items: (key tile, head, instance)
@@ -136,6 +137,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint64_t* bar_s = bars + 3;
     uint64_t* bar_g = bars + 4;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+    uint64_t* bar_acc = bars + 6;                   // every product of the item complete: dV, dK final, operands free
     float* s_stat = reinterpret_cast<float*>(smem_dyn + 64);      // [2 stages][128] lse of the query tile, log2 domain
     float* s_dpart = s_stat + 2 * kTile;                          // [2 halves][128] partial Delta = sum over 32 head dims of dO O
     unsigned char* sK = align_tiles(smem_dyn + 64 + 4 * kTile * sizeof(float));
@@ -144,7 +146,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     unsigned char* sdO = sQ + 2 * kTileBytes;       // 2 stages
     unsigned char* sPt = sdO + 2 * kTileBytes;      // P^T  : rows = keys, columns = queries (two 64-query panels)
     unsigned char* sdSt = sPt + 2 * kTileBytes;     // dS^T : same shape
-    if (sdSt + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
+    unsigned char* sDQ = sdSt + 2 * kTileBytes;     // dQ_i as fp32: panel `half` = head dimensions 32 half .. 32 half + 31, 128-byte swizzled rows
+    if (sDQ + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
         if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
         return;
     }
@@ -162,11 +165,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         mbar_init(bar_qdo + 1, 1);
         mbar_init(bar_s, 1);
         mbar_init(bar_g, 1);
+        mbar_init(bar_acc, 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v);
         tma_prefetch_desc(&map_do);
+        tma_prefetch_desc(&map_acc);
     }
     tc_fence_before();
     __syncthreads();
@@ -251,12 +256,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             const uint32_t st = q_count & 1, ph = q_count & 1;
             float next_lse = 0.f;
             if (i + 1 < n_q) {
-                if (warp == 0) {                         // the other stage was released by the wait on bar_g of the previous tile
-                    if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);
-                    __syncwarp();
-                    load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), P.src, (i + 1) * kTile, n_sel, h, b, P.H);
-                    load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), P.src_do, (i + 1) * kTile, n_sel, h, b, P.H);
-                }
                 next_lse = load_lse(b, h, (i + 1) * kTile + row);        // both land while this tile is processed
                 dl_next = load_delta(b, h, (i + 1) * kTile + row);
                 if (!use_delta) load_o(b, h, (i + 1) * kTile + row, o_next);
@@ -281,6 +280,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             __syncthreads();                             // row statistics of this stage visible
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
+            if (warp == 0 && i + 1 < n_q) {              // scores of this tile done => every product of the previous tile is done:
+                if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);      // the other Q / dO stage is free
+                __syncwarp();
+                load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), P.src, (i + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), P.src_do, (i + 1) * kTile, n_sel, h, b, P.H);
+            }
 
             // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
             const float* lse2 = s_stat + st * kTile + half * 64;
@@ -312,11 +317,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             }
             fence_proxy_async_smem();
             tc_fence_before();
+            if (tid == 0) bulk_wait_group_read0();       // the previous tile's dQ reduction has read its shared-memory tile
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
                 const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ + st * kTileBytes), d0 = smem_u32(sdO + st * kTileBytes),
                                k0 = smem_u32(sK);
+#pragma unroll
+                for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K, first: it is drained
+                    tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
+                                idesc_mnmn, ks > 0);                 // while the other products and the next scores run
+                tc_commit(bar_g);
 #pragma unroll
                 for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
                     const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
@@ -325,11 +336,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_mma_bf16(tm_dk, umma_desc_sw128(dst + a_off, 16, 1024), umma_desc_sw128(q0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
                                 (i > 0) | (ks > 0));
                 }
-#pragma unroll
-                for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K
-                    tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
-                                idesc_mnmn, ks > 0);
-                tc_commit(bar_g);
+                if (i + 1 == n_q) tc_commit(bar_acc);
                 if (i + 1 < n_q) {                       // S^T, dP^T of the next query tile queue up behind these products
                     ok &= mbar_wait(bar_qdo + (st ^ 1), ((q_count + 1) >> 1) & 1);
                     tc_fence_after();
@@ -362,17 +369,26 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                 make_uint4(pack2(dqv[8 * q + 0] * P.scale, dqv[8 * q + 1] * P.scale), pack2(dqv[8 * q + 2] * P.scale, dqv[8 * q + 3] * P.scale),
                                            pack2(dqv[8 * q + 4] * P.scale, dqv[8 * q + 5] * P.scale), pack2(dqv[8 * q + 6] * P.scale, dqv[8 * q + 7] * P.scale));
                     }
-                } else if (qv) {
-                    float* dst = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + qrow) * P.H + h) * kDP + half * 32;
+                } else {                                 // rows past n_sel are exact zeros (their probabilities are zero)
+                    unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
 #pragma unroll
-                    for (int x = 0; x < 32; x += 4) red_add_f32x4(dst + x, dqv[x], dqv[x + 1], dqv[x + 2], dqv[x + 3]);
+                    for (int x = 0; x < 8; ++x)
+                        *reinterpret_cast<float4*>(rowp + ((x ^ (row & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
+                    fence_proxy_async_smem();
                 }
             }
             tc_fence_before();
             ok = __syncthreads_and(ok);
             if (!ok) break;
+            if (!single_tile && tid == 0) {              // one bulk reduce-add per half: dq_acc[b, 128 i .., h, 32 half ..] += tile
+                tma_reduce_add_4d(&map_acc, sDQ, 0, h, i * kTile, b);
+                tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, h, i * kTile, b);
+                bulk_commit_group();
+            }
         }
 
+        ok &= mbar_wait(bar_acc, n_done & 1);
+        tc_fence_after();
         {   // dV, dK of this key tile: every thread takes part in the warp-collective loads, only valid key rows store
             const bool store = ok && key_valid && half * 32 < P.D;
             const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
@@ -401,6 +417,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
     }
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
+    if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
@@ -494,6 +511,8 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         if (int st = make_tile_map(&mv, v, c.B, c.N, c.N, c.H)) return st;
         if (int st = make_tile_map(&mdo, d_o, c.B, c.N, c.N, c.H)) return st;
     }
+    CUtensorMap macc;
+    if (int st = make_acc_map(&macc, base + w.dq_acc, c.B, w.Ncap, c.H)) return st;
     BwdParams P{};
     P.lse = lse; P.o = static_cast<const __nv_bfloat16*>(o); P.delta = pre_delta ? reinterpret_cast<const float*>(base + w.delta) : nullptr;
     P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
@@ -516,7 +535,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
         const int grid = static_cast<int>(worst < sm_count() ? worst : sm_count());      // one CTA per SM (all of tensor memory)
         LaunchScope ls_(K_ATTN_BWD, stream);
-        attn_bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, P);
+        attn_bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, macc, P);
     }
     if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
 

@@ -43,6 +43,10 @@ inline AttnWs attn_layout(const vardrop_attn_cfg& c) {
 // 128-byte swizzle, rows outside the tensor read as zero.
 int make_row_map(CUtensorMap* map, const void* base, long long rows);
 
+// Tensor map over the fp32 dQ' accumulator [B, Ncap, H, 64]: box = 128 tokens x 32 floats (one 128-byte swizzled row
+// per token) of one head, the unit of the backward kernel's bulk reduce-add.
+int make_acc_map(CUtensorMap* map, const void* base, int B, int Ncap, int H);
+
 // Number of SMs of the current device (cached per thread and device).
 int sm_count();
 

@@ -70,6 +70,19 @@ int make_row_map(CUtensorMap* map, const void* base, long long rows) {
     return VARDROP_OK;
 }
 
+int make_acc_map(CUtensorMap* map, const void* base, int B, int Ncap, int H) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(kDP), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(Ncap), static_cast<cuuint64_t>(B)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kDP) * 4, static_cast<cuuint64_t>(H) * kDP * 4, static_cast<cuuint64_t>(Ncap) * H * kDP * 4};
+    const cuuint32_t box[4] = {32, 1, kTile, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled (accumulator) failed with code %d", static_cast<int>(r));
+    return VARDROP_OK;
+}
+
 int attn_validate(const vardrop_attn_cfg& c) {
     if (c.B < 1 || c.N < 1 || c.H < 1) return fail(VARDROP_ERR_INVALID_ARG, "attention: B, N, H >= 1 required (B=%d N=%d H=%d)", c.B, c.N, c.H);
     if (c.D != 32 && c.D != 64) return fail(VARDROP_ERR_UNSUPPORTED, "attention: head dimension %d (32 or 64 supported)", c.D);
