@@ -23,11 +23,6 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
     return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w));
 }
 
-// four consecutive floats added to global memory in one 16-byte reduction
-__device__ __forceinline__ void red_add_f32x4(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
 // ---------------------------------------------------------------------------------------------------------
 // prep
 // ---------------------------------------------------------------------------------------------------------
@@ -194,15 +189,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
     const bool use_delta = P.delta != nullptr && n_q > 1;      // precomputed Delta exists only when there are several key tiles
 
-    // S^T = K Q^T and dP^T = V dO^T of one query tile (issued by one thread), completion on bar_s
-    auto issue_scores = [&](const unsigned char* q_tile, const unsigned char* do_tile) {
-        const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV), q0 = smem_u32(q_tile), d0 = smem_u32(do_tile);
+    // operand descriptors, built once and stepped by additions: K-major views for the scores and the P^T / dS^T panels,
+    // MN-major views where the reduction runs over the rows of the tile
+    const uint64_t d_k = umma_desc_sw128(smem_u32(sK), 16, 1024), d_v = umma_desc_sw128(smem_u32(sV), 16, 1024);
+    const uint64_t d_q0 = umma_desc_sw128(smem_u32(sQ), 16, 1024), d_do0 = umma_desc_sw128(smem_u32(sdO), 16, 1024);
+    const uint64_t d_pt = umma_desc_sw128(smem_u32(sPt), 16, 1024), d_dst = umma_desc_sw128(smem_u32(sdSt), 16, 1024);
+    const uint64_t m_q0 = umma_desc_sw128(smem_u32(sQ), kTileBytes, 1024), m_do0 = umma_desc_sw128(smem_u32(sdO), kTileBytes, 1024);
+    const uint64_t m_dst = umma_desc_sw128(smem_u32(sdSt), kTileBytes, 1024), m_k = umma_desc_sw128(smem_u32(sK), kTileBytes, 1024);
+    // S^T = K Q^T and dP^T = V dO^T of the query tile in ring stage `stage` (issued by one thread), completion on bar_s
+    auto issue_scores = [&](uint32_t stage) {
+        const uint64_t dq_ = umma_desc_advance(d_q0, stage * kTileBytes), dd_ = umma_desc_advance(d_do0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
-            tc_mma_bf16(tm_st, umma_desc_sw128(k0 + ks * 32, 16, 1024), umma_desc_sw128(q0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+            tc_mma_bf16(tm_st, umma_desc_advance(d_k, ks * 32), umma_desc_advance(dq_, ks * 32), idesc_kk, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
-            tc_mma_bf16(tm_dpt, umma_desc_sw128(v0 + ks * 32, 16, 1024), umma_desc_sw128(d0 + ks * 32, 16, 1024), idesc_kk, ks > 0);
+            tc_mma_bf16(tm_dpt, umma_desc_advance(d_v, ks * 32), umma_desc_advance(dd_, ks * 32), idesc_kk, ks > 0);
         tc_commit(bar_s);
     };
 
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 ok &= mbar_wait(bar_kv, n_done & 1);
                 ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
                 tc_fence_after();
-                issue_scores(sQ + st * kTileBytes, sdO + st * kTileBytes);
+                issue_scores(st);
             }
             if (use_delta) {
                 s_dpart[half * kTile + row] = dl_cur;    // half 1 holds the value, half 0 contributes zero
@@ -321,26 +323,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
-                const uint32_t pt = smem_u32(sPt), dst = smem_u32(sdSt), q0 = smem_u32(sQ + st * kTileBytes), d0 = smem_u32(sdO + st * kTileBytes),
-                               k0 = smem_u32(sK);
+                const uint64_t mq = umma_desc_advance(m_q0, st * kTileBytes), mdo = umma_desc_advance(m_do0, st * kTileBytes);
 #pragma unroll
                 for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K, first: it is drained
-                    tc_mma_bf16(tm_dq, umma_desc_sw128(dst + ks * 2048, kTileBytes, 1024), umma_desc_sw128(k0 + ks * 2048, kTileBytes, 1024),
-                                idesc_mnmn, ks > 0);                 // while the other products and the next scores run
-                tc_commit(bar_g);
+                    tc_mma_bf16(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
+                tc_commit(bar_g);                                    // while the other products and the next scores run
+                const uint32_t acc_on = i > 0;
 #pragma unroll
                 for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
                     const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
-                    tc_mma_bf16(tm_dv, umma_desc_sw128(pt + a_off, 16, 1024), umma_desc_sw128(d0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
-                                (i > 0) | (ks > 0));
-                    tc_mma_bf16(tm_dk, umma_desc_sw128(dst + a_off, 16, 1024), umma_desc_sw128(q0 + ks * 2048, kTileBytes, 1024), idesc_kmn,
-                                (i > 0) | (ks > 0));
+                    tc_mma_bf16(tm_dv, umma_desc_advance(d_pt, a_off), umma_desc_advance(mdo, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
+                    tc_mma_bf16(tm_dk, umma_desc_advance(d_dst, a_off), umma_desc_advance(mq, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
                 }
                 if (i + 1 == n_q) tc_commit(bar_acc);
                 if (i + 1 < n_q) {                       // S^T, dP^T of the next query tile queue up behind these products
                     ok &= mbar_wait(bar_qdo + (st ^ 1), ((q_count + 1) >> 1) & 1);
                     tc_fence_after();
-                    issue_scores(sQ + (st ^ 1) * kTileBytes, sdO + (st ^ 1) * kTileBytes);
+                    issue_scores(st ^ 1);
                 }
             }
             if (i + 1 < n_q) {

@@ -162,6 +162,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
     d |= 2ull << 61;                                                    // layout: 128-byte swizzle
     return d;
 }
+// The same descriptor `bytes` further into the tile (a multiple of 16; the start-address field counts 16-byte units).
+// Building a descriptor takes a dozen integer instructions and a single thread issues every product, so kernels build
+// one descriptor per operand tile and step it with this addition.
+__device__ __forceinline__ uint64_t umma_desc_advance(uint64_t desc, uint32_t bytes) { return desc + (bytes >> 4); }
+
 // Instruction descriptor: bf16 x bf16 -> fp32, dense, M x N tile; a_mn / b_mn = 1 selects an MN-major operand.
 __device__ __host__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn, int b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
