@@ -167,13 +167,14 @@ int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, i
  *   lse_i = log sum_j exp(S_ij).
  * bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before the second product.
  *
- * cfg (host)  B, N, H, D (D = 32 or 64; N <= 65536), sm_scale (0 selects 1/sqrt(D)).
+ * cfg (host)  B, N, H, D (D = 32 or 64; N <= 65536), sm_scale (0 selects 1/sqrt(D)), S (1 or B).
  * q, k, v     [B, N, H, D] bf16, contiguous.
- * sel_idx     [N] int32, ascending kept variates (row 0 of vardrop_select's output), or NULL for the
+ * sel_idx     [S, N] int32, ascending kept variates (vardrop_select's output: S = 1 for the paper's batch-wise
+ *             grouping, S = B when every instance was hashed and sampled on its own), or NULL for the
  *             all-token path (VarDrop off, the inference / "ground" configuration of the paper).
- * n_sel       [1] int32 on the device, number of valid entries of sel_idx; ignored when sel_idx is NULL.
- * o           [B, N, H, D] bf16 out; rows 0..n_sel-1 of every instance hold O', the rest is untouched.
- * lse         [B, H, N] float32 out; entries 0..n_sel-1 valid.
+ * n_sel       [S] int32 on the device, number of valid entries of each row of sel_idx; ignored when sel_idx is NULL.
+ * o           [B, N, H, D] bf16 out; rows 0..n_sel[s(b)]-1 of instance b hold O', the rest is untouched.
+ * lse         [B, H, N] float32 out; entries 0..n_sel[s(b)]-1 valid.
  * ws          scratch of vardrop_attn_workspace_bytes.  After the call it holds what the backward pass of the same
  *             step needs (staged Q', K', V' where the library stages them, a cleared dQ' accumulator):
  *             vardrop_attn_bwd must be given the same, unmodified workspace, once per forward call.
@@ -181,6 +182,7 @@ int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, i
 typedef struct {
     int32_t B, N, H, D;
     float sm_scale;
+    int32_t S;      /* selections: 0 or 1 = one shared by all instances (batch-wise grouping), B = one per instance */
 } vardrop_attn_cfg;
 
 size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg);
@@ -198,7 +200,7 @@ int vardrop_attn_fwd(const void* q, const void* k, const void* v, const int32_t*
  * q, k, v, sel_idx, n_sel, cfg, ws   as given to vardrop_attn_fwd (ws unmodified since).
  * o, lse      outputs of vardrop_attn_fwd.
  * d_o         [B, N, H, D] bf16, gradient of o; rows 0..n_sel-1 are read.
- * inv_idx     [N] int32 from vardrop_select (NULL when sel_idx is NULL).
+ * inv_idx     [S, N] int32 from vardrop_select (NULL when sel_idx is NULL).
  * dq, dk, dv  [B, N, H, D] bf16 out, full variate layout.
  * dQ' is accumulated across key tiles with fp32 atomic adds, so its low-order bits may differ from run
  * to run; dK', dV' are bit-reproducible.

@@ -30,7 +30,7 @@ class SelectCfg(C.Structure):
 
 
 class AttnCfg(C.Structure):
-    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float)]
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float), ("S", C.c_int32)]
 
 
 class VardropError(RuntimeError):

@@ -32,16 +32,16 @@ struct PrepParams {
     uint4* dog;           // [B, Ncap, H, 64] bf16 staged dO (NULL: not needed)
     float* delta;         // [B, H, Ncap]
     float4* dq_acc;       // [B, Ncap, H, 64] fp32
-    const int32_t* n_sel; // NULL: N
-    int N, Ncap, H, D;
+    const int32_t* n_sel; // [S] kept counts; NULL: N
+    int N, Ncap, H, D, S;
 };
 
 // one thread per 16-byte chunk of a staged (token, head) row; the 8 threads of a row reduce Delta by shuffles
 __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
-    const int n_sel = P.n_sel ? *P.n_sel : P.N;
+    const int b = blockIdx.y;
+    const int n_sel = P.n_sel ? P.n_sel[P.S > 1 ? b : 0] : P.N;
     if (!P.dog && n_sel <= kTile) return;            // a single key tile: the main kernel computes Delta itself
     const int n_fill = min(P.Ncap, (n_sel + kTile - 1) / kTile * kTile);
-    const int b = blockIdx.y;
     const int chunks_row = P.H * 8;
     const int src_chunks_head = P.D / 8;
     const int total = n_fill * chunks_row;            // a multiple of 8; blockDim is a multiple of 8
@@ -84,10 +84,10 @@ struct BwdParams {
     __nv_bfloat16* dq;      // [B, N, H, D]; written here only when there is a single key tile
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
-    const int32_t* sel_idx; // NULL: identity
-    const int32_t* n_sel;   // NULL: N
+    const int32_t* sel_idx; // [S, N]; NULL: identity
+    const int32_t* n_sel;   // [S]; NULL: N
     int* status;
-    int B, N, Ncap, H, D;
+    int B, N, Ncap, H, D, S;
     float scale, scale_log2;
 };
 
@@ -120,12 +120,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                                                    const __grid_constant__ CUtensorMap map_v,
                                                                    const __grid_constant__ CUtensorMap map_do,
                                                                    const __grid_constant__ CUtensorMap map_acc, const BwdParams P) {
-    const int n_sel = P.n_sel ? *P.n_sel : P.N;
-    const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles
-    const int n_items = n_q * P.H * P.B;                       // work items: (key tile, head, instance)
+    extern __shared__ unsigned char smem_dyn[];
+    const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
     if (static_cast<int>(blockIdx.x) >= n_items) return;
 
-    extern __shared__ unsigned char smem_dyn[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
     uint64_t* bar_kv = bars + 0;
     uint64_t* bar_qdo = bars + 1;                   // [2]
@@ -183,11 +182,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major, B MN-major, N = 64
     constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
 
+    int n_sel = P.N;            // kept tokens of the instance being processed (set per work item)
+    bool use_delta = false;     // precomputed Delta in use for this instance
     bool ok = true;
     uint32_t q_count = 0;       // query tiles consumed so far by this CTA: stage = q_count & 1
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
-    const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
-    const bool use_delta = P.delta != nullptr && n_q > 1;      // precomputed Delta exists only when there are several key tiles
 
     // operand descriptors, built once and stepped by additions: K-major views for the scores and the P^T / dS^T panels,
     // MN-major views where the reduction runs over the rows of the tile
@@ -231,10 +230,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         return a0.x * g0.x + a0.y * g0.y + a1.x * g1.x + a1.y * g1.y + a2.x * g2.x + a2.y * g2.y + a3.x * g3.x + a3.y * g3.y;
     };
 
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
-        const int jt = item % n_q;
-        const int h = (item / n_q) % P.H;
-        const int b = item / (n_q * P.H);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int jt = item % n_t_max;
+        const int h = (item / n_t_max) % P.H;
+        const int b = item / (n_t_max * P.H);
+        const int srow = P.S > 1 ? b : 0;
+        n_sel = P.n_sel ? P.n_sel[srow] : P.N;
+        const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
+        if (jt >= n_q) continue;
+        const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
+        use_delta = P.delta != nullptr && n_q > 1;                 // precomputed Delta exists only when there are several key tiles
+        const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
+        TileSource src = P.src, src_do = P.src_do;
+        if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
         if (warp == 0) {            // every MMA of the previous item has completed: K, V and both Q/dO stages are free
             const uint32_t st0 = q_count & 1;
             if (tid == 0) {
@@ -242,10 +250,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
             }
             __syncwarp();
-            load_tile(sK, &map_k, bar_kv, P.src, jt * kTile, n_sel, h, b, P.H);
-            load_tile(sV, &map_v, bar_kv, P.src, jt * kTile, n_sel, h, b, P.H);
-            load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, P.src, 0, n_sel, h, b, P.H);
-            load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, P.src_do, 0, n_sel, h, b, P.H);
+            load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, src, 0, n_sel, h, b, P.H);
+            load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, src_do, 0, n_sel, h, b, P.H);
         }
         if (half == 0) s_stat[(q_count & 1) * kTile + row] = load_lse(b, h, row);
         uint4 o_cur[4], o_next[4];
@@ -285,8 +293,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (warp == 0 && i + 1 < n_q) {              // scores of this tile done => every product of the previous tile is done:
                 if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);      // the other Q / dO stage is free
                 __syncwarp();
-                load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), P.src, (i + 1) * kTile, n_sel, h, b, P.H);
-                load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), P.src_do, (i + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), src, (i + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), src_do, (i + 1) * kTile, n_sel, h, b, P.H);
             }
 
             // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
@@ -360,7 +368,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tmem_ld_wait();
                 if (single_tile) {                       // final value: straight to the full-layout gradient, scaled, bf16
                     if (qv && half * 32 < P.D) {
-                        const int n = P.sel_idx ? P.sel_idx[qrow] : qrow;
+                        const int n = sel ? sel[qrow] : qrow;
                         __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
@@ -390,7 +398,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         tc_fence_after();
         {   // dV, dK of this key tile: every thread takes part in the warp-collective loads, only valid key rows store
             const bool store = ok && key_valid && half * 32 < P.D;
-            const int n = store ? (P.sel_idx ? P.sel_idx[key] : key) : 0;
+            const int n = store ? (sel ? sel[key] : key) : 0;
             const size_t out = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
             float acc[32];
             tmem_ld32(tm_dv + lane_sel + half * 32, acc);
@@ -414,6 +422,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             tc_fence_before();
             __syncthreads();        // the accumulators are read out before the next item's products overwrite them
         }
+        ++n_done;
     }
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
@@ -428,15 +437,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 struct FinishParams {
     const float4* dq_acc;    // [B, Ncap, H, 64] fp32
     uint4 *dq, *dk, *dv;     // [B, N, H, D] bf16
-    const int32_t* inv_idx;  // NULL: identity
-    const int32_t* n_sel;    // NULL: N
-    int N, Ncap, H, D;
+    const int32_t* inv_idx;  // [S, N]; NULL: identity
+    const int32_t* n_sel;    // [S]; NULL: N
+    int N, Ncap, H, D, S;
     float scale;
 };
 
 __global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
     const int b = blockIdx.y;
-    const bool dq_done = (P.n_sel ? *P.n_sel : P.N) <= kTile;     // single key tile: the main kernel wrote the kept dq rows
+    const int srow = P.S > 1 ? b : 0;
+    const int32_t* inv = P.inv_idx ? P.inv_idx + static_cast<size_t>(srow) * P.N : nullptr;
+    const bool dq_done = (P.n_sel ? P.n_sel[srow] : P.N) <= kTile;      // single key tile: the main kernel wrote the kept dq rows
     const int chunks_head = P.D / 8;
     const int chunks_row = P.H * chunks_head;
     const int total = P.N * chunks_row;
@@ -444,7 +455,7 @@ __global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
         const int n = idx / chunks_row;
         const int c = idx - n * chunks_row;
         const int h = c / chunks_head, dc = c - h * chunks_head;
-        const int j = P.inv_idx ? P.inv_idx[n] : n;
+        const int j = inv ? inv[n] : n;
         const size_t dst = static_cast<size_t>(b) * total + idx;
         if (j >= 0) {
             if (dq_done) continue;
@@ -483,7 +494,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         R.delta = pre_delta ? reinterpret_cast<float*>(base + w.delta) : nullptr;
         R.dq_acc = nullptr;
         R.n_sel = sel_idx ? n_sel : nullptr;
-        R.N = c.N; R.Ncap = w.Ncap; R.H = c.H; R.D = c.D;
+        R.N = c.N; R.Ncap = w.Ncap; R.H = c.H; R.D = c.D; R.S = attn_sel_rows(c);
         const long long work = static_cast<long long>(w.Ncap) * c.H * 8;
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 4 * sm_count() / c.B);              // about four CTAs per SM in total
@@ -521,7 +532,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     P.dq = static_cast<__nv_bfloat16*>(dq); P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
     P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);
-    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
+    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D; P.S = attn_sel_rows(c);
     P.scale = scale; P.scale_log2 = scale * 1.4426950408889634f;
     static thread_local int attr_dev = -1;
     int dev = 0;
@@ -543,7 +554,7 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     F.dq = static_cast<uint4*>(dq); F.dk = static_cast<uint4*>(dk); F.dv = static_cast<uint4*>(dv);
     F.inv_idx = sel_idx ? inv_idx : nullptr;
     F.n_sel = sel_idx ? n_sel : nullptr;
-    F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.scale = scale;
+    F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.S = attn_sel_rows(c); F.scale = scale;
     {
         const long long work = static_cast<long long>(c.N) * c.H * (c.D / 8);
         int gx = static_cast<int>((work + 255) / 256);

@@ -63,7 +63,7 @@ __device__ __forceinline__ unsigned char* align_tiles(unsigned char* p) {
 //            (idx = NULL: the slot itself) while tok0 + j < n_valid, and a row past the end (zeros) otherwise.
 // Called by all 32 lanes of one warp; `lane0_expect` bytes are announced on the barrier by lane 0 first.
 struct TileSource {
-    const int32_t* idx;    // gather indices (NULL: identity)
+    const int32_t* idx;    // gather indices of the instance's selection (NULL: identity)
     int gathered;          // 0: tiled box, 1: row gathers
     int tokens;            // tokens per instance in the gathered tensor
     int rows_total;        // B * tokens * H
@@ -94,6 +94,21 @@ __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap*
 //            zero-padded to 64 there; or a selection at large N, where every tile is re-read many times and
 //            contiguous, L2-resident tiles pay for the extra pass)
 constexpr int kGatherMaxN = 512;
+// Number of selection rows: one shared by the batch, or one per instance.
+inline int attn_sel_rows(const vardrop_attn_cfg& c) { return c.S > 1 ? c.S : 1; }
+
+// Largest kept count over the selection rows (device, whole CTA; `scratch` is one int of shared memory).
+__device__ __forceinline__ int max_kept(const int32_t* n_sel, int S, int N, int* scratch) {
+    if (!n_sel) return N;
+    if (threadIdx.x == 0) *scratch = 0;
+    __syncthreads();
+    int m = 0;
+    for (int s = threadIdx.x; s < S; s += blockDim.x) m = max(m, n_sel[s]);
+    if (m > 0) atomicMax(scratch, m);
+    __syncthreads();
+    return *scratch;
+}
+
 inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D != kDP || (sel_idx != nullptr && c.N > kGatherMaxN); }
 inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D == kDP && sel_idx != nullptr && c.N <= kGatherMaxN; }
 

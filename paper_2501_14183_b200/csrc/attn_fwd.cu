@@ -89,6 +89,7 @@ int attn_validate(const vardrop_attn_cfg& c) {
     if (c.N > 65536) return fail(VARDROP_ERR_UNSUPPORTED, "attention: N=%d above 65536", c.N);
     if (static_cast<long long>(c.B) * c.N * c.H >= (1ll << 31)) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B*N*H above 2^31");
     if (c.H > 65535 || c.B > 65535) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B or H above 65535");
+    if (c.S != 0 && c.S != 1 && c.S != c.B) return fail(VARDROP_ERR_INVALID_ARG, "attention: S=%d must be 1 (shared selection) or B (one per instance)", c.S);
     if (!(c.sm_scale >= 0.f)) return fail(VARDROP_ERR_INVALID_ARG, "attention: sm_scale must be >= 0 (0 selects 1/sqrt(D))");
     return VARDROP_OK;
 }
@@ -105,15 +106,17 @@ struct GatherParams {
     uint4* dst[3];
     const int32_t* sel_idx;   // NULL: identity
     const int32_t* n_sel;     // NULL with sel_idx NULL
-    int N, Ncap, H, D;
+    int N, Ncap, H, D, S;     // S selection rows (1: shared, B: per instance)
 };
 
 __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
-    const int n_sel = P.sel_idx ? *P.n_sel : P.N;
+    const int b = blockIdx.y, t = blockIdx.z;
+    const int srow = P.S > 1 ? b : 0;                                         // selection row of this instance
+    const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
+    const int n_sel = P.sel_idx ? P.n_sel[srow] : P.N;
     const int n_fill = min(P.Ncap, (n_sel + kTile - 1) / kTile * kTile);     // rows to define: kept + zero tail of the tile
     const int chunks_row = P.H * (kDP / 8);                                   // 16-byte chunks per staged token
     const int src_chunks_head = P.D / 8;
-    const int b = blockIdx.y, t = blockIdx.z;
     const int total = n_fill * chunks_row;
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int j = idx / chunks_row;
@@ -121,7 +124,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
         const int h = c / (kDP / 8), dc = c - h * (kDP / 8);
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
         if (j < n_sel && dc < src_chunks_head) {
-            const int n = P.sel_idx ? P.sel_idx[j] : j;
+            const int n = sel ? sel[j] : j;
             val = __ldg(P.src[t] + (static_cast<size_t>(b) * P.N + n) * (P.H * src_chunks_head) + h * src_chunks_head + dc);
         }
         P.dst[t][(static_cast<size_t>(b) * P.Ncap + j) * chunks_row + c] = val;
@@ -134,11 +137,11 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
 struct FwdParams {
     __nv_bfloat16* o;
     float* lse;
-    const int32_t* n_sel;   // NULL: all N tokens
+    const int32_t* n_sel;   // [S] kept counts; NULL: all N tokens
     int* status;
     float4* dq_acc;         // [B, Ncap, H, 64] fp32: zeroed here for the backward pass when it will accumulate into it
     TileSource src;         // where Q, K, V tiles come from
-    int B, N, Ncap, H, D;
+    int B, N, Ncap, H, D, S;
     float scale_log2;       // sm_scale * log2(e)
 };
 
@@ -174,12 +177,11 @@ __device__ __forceinline__ void store_row_chunk32(unsigned char* tile, int r, in
 __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                 const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v, const FwdParams P) {
-    const int n_sel = P.n_sel ? *P.n_sel : P.N;
-    const int n_kv = (n_sel + kTile - 1) / kTile;              // key tiles = query tiles
-    const int n_items = n_kv * P.H * P.B;                      // work items: (query tile, head, instance)
+    extern __shared__ unsigned char smem_dyn[];
+    const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_items = n_t_max * P.H * P.B;                   // work items: (query tile, head, instance); short instances skip tiles
     if (static_cast<int>(blockIdx.x) >= n_items) return;
 
-    extern __shared__ unsigned char smem_dyn[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);     // barriers and the TMEM slot sit in front of the tiles
     uint64_t* bar_q = bars + 0;
     uint64_t* bar_kv = bars + 1;                    // [2]
@@ -234,10 +236,16 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
     uint32_t kv_count = 0;      // K/V tiles consumed so far by this CTA: ring stage and barrier phase follow from it
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_q)
 
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n_done) {
-        const int qt = item % n_kv;
-        const int h = (item / n_kv) % P.H;
-        const int b = item / (n_kv * P.H);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int qt = item % n_t_max;
+        const int h = (item / n_t_max) % P.H;
+        const int b = item / (n_t_max * P.H);
+        const int srow = P.S > 1 ? b : 0;
+        const int n_sel = P.n_sel ? P.n_sel[srow] : P.N;       // kept tokens of this instance
+        const int n_kv = (n_sel + kTile - 1) / kTile;          // its key tiles = query tiles
+        if (qt >= n_kv) continue;
+        TileSource src = P.src;
+        if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
         if (warp == 0) {            // every MMA of the previous item has completed: Q and both ring stages are free
             const uint32_t st0 = kv_count & 1;
             if (tid == 0) {
@@ -245,9 +253,9 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                 mbar_expect_tx(bar_kv + st0, 2 * kTileBytes);
             }
             __syncwarp();
-            load_tile(sQ, &map_q, bar_q, P.src, qt * kTile, n_sel, h, b, P.H);
-            load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, P.src, 0, n_sel, h, b, P.H);
-            load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, P.src, 0, n_sel, h, b, P.H);
+            load_tile(sQ, &map_q, bar_q, src, qt * kTile, n_sel, h, b, P.H);
+            load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, src, 0, n_sel, h, b, P.H);
+            load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, src, 0, n_sel, h, b, P.H);
         }
         if (n_kv > 1) {             // the backward pass will add per-key-tile pieces of dQ' into the accumulator: clear this tile's rows
 #pragma unroll
@@ -268,8 +276,8 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
             if (warp == 0 && j + 1 < n_kv) {             // the other stage was released by the wait on bar_o of the previous tile
                 if (tid == 0) mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
                 __syncwarp();
-                load_tile(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), P.src, (j + 1) * kTile, n_sel, h, b, P.H);
-                load_tile(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), P.src, (j + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
+                load_tile(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
             }
             if (tid == 0) {
                 if (j == 0) {                            // later tiles: issued right behind the previous tile's P V
@@ -363,6 +371,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
             }
             P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
+        ++n_done;
     }
 
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
@@ -386,7 +395,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         G.dst[0] = reinterpret_cast<uint4*>(base + w.qg); G.dst[1] = reinterpret_cast<uint4*>(base + w.kg);
         G.dst[2] = reinterpret_cast<uint4*>(base + w.vg);
         G.sel_idx = sel_idx; G.n_sel = sel_idx ? n_sel : nullptr;
-        G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D;
+        G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D; G.S = attn_sel_rows(c);
         const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 4 * sm_count() / (3 * c.B));        // about four CTAs per SM in total; each strides over its rows
@@ -412,7 +421,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
     P.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
     P.src.idx = sel_idx; P.src.gathered = attn_uses_gather(c, sel_idx) ? 1 : 0; P.src.tokens = c.N;
     P.src.rows_total = c.B * c.N * c.H;
-    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D;
+    P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D; P.S = attn_sel_rows(c);
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
     P.scale_log2 = scale * 1.4426950408889634f;
     static thread_local int attr_dev = -1;

@@ -112,3 +112,43 @@ def test_attention_argument_errors():
     with pytest.raises(vd.VardropError) as e:
         vd.vardrop_attn_fwd(q, None, q, None, None, vd.AttnCfg(1, 8, 1, 64, 0.0), q, lse, ws)
     assert e.value.status == vd.ERR_INVALID_ARG
+
+
+def test_attention_per_instance_selections():
+    """One selection per instance (S = B): every instance keeps its own variates, with different counts, spanning one and two tiles."""
+    B, N, H, D = 4, 300, 2, 64
+    dev, ref = bf16_tokens(B, N, H, D, 1.0, seed=21)
+    q, k, v, d_full = dev
+    counts = [17, 128, 129, 260]
+    sels = [pick(N, c, seed=100 + i) for i, c in enumerate(counts)]
+    sel_pad = np.full((B, N), -1, np.int32); inv = np.full((B, N), -1, np.int32)
+    for b, s_ in enumerate(sels):
+        sel_pad[b, :len(s_)] = s_
+        inv[b, s_] = np.arange(len(s_), dtype=np.int32)
+    cfg = vd.AttnCfg(B, N, H, D, 0.0, B)
+    ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
+    ws.view(torch.int16).fill_(0x7FC1)
+    nan = float("nan")
+    o = torch.full((B, N, H, D), nan, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, H, N), nan, dtype=torch.float32, device="cuda")
+    d_o = torch.full((B, N, H, D), nan, dtype=torch.bfloat16, device="cuda")
+    for b, c in enumerate(counts):
+        d_o[b, :c] = d_full[b, :c]
+    sel_t, inv_t = torch.from_numpy(sel_pad).cuda(), torch.from_numpy(inv).cuda()
+    nsel_t = torch.tensor(counts, dtype=torch.int32, device="cuda")
+    vd.vardrop_attn_fwd(q, k, v, sel_t, nsel_t, cfg, o, lse, ws)
+    dq, dk, dv = (torch.full((B, N, H, D), nan, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, sel_t, nsel_t, inv_t, cfg, dq, dk, dv, ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.OK
+    for b, (c, s_) in enumerate(zip(counts, sels)):
+        cut = [r[b:b + 1] for r in ref]
+        wo, wl = oracle.attn_fwd(cut[0], cut[1], cut[2], s_)
+        assert_attn_close(o[b:b + 1, :c].double().cpu().numpy(), wo, f"o[{b}]")
+        assert_attn_close(lse[b:b + 1, :, :c].double().cpu().numpy(), wl, f"lse[{b}]")
+        wq, wk, wv = oracle.attn_bwd(cut[0], cut[1], cut[2], cut[3][:, :c], s_)
+        for got, want, name in ((dq, wq, "dq"), (dk, wk, "dk"), (dv, wv, "dv")):
+            g = got[b:b + 1].double().cpu().numpy()
+            assert_attn_close(g, want, f"{name}[{b}]")
+            assert np.all(g[:, np.setdiff1d(np.arange(N), s_)] == 0.0)
+        assert torch.isnan(o[b, c:].float()).all()

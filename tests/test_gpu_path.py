@@ -87,3 +87,45 @@ def test_vardrop_off_full_attention(name, pairs):
     toks = inputs.make_tokens(w.B, w.N, w.H, w.D, w.qkv_std, seed=w.seed + 1)
     dev, _, o, lse, dq, dk, dv = run_path(w, None, toks, vardrop=False)
     check_attention_samples(w, dev, None, o, lse, dq, dk, dv, pairs)
+
+
+def test_whole_path_per_instance_scope():
+    """Every instance hashed, grouped and sampled on its own (hash scope 1, S = B selections) and attended with its own
+    kept set: the algorithm of the paper run with batch size one per instance."""
+    w = inputs.WORKLOADS["elec"]
+    B = 6
+    x, okeys, _, _, _ = gap_filtered_windows(inputs.make_windows(w, B=B), w.k, scope=1)
+    toks = inputs.make_tokens(B, w.N, w.H, w.D, w.qkv_std, seed=5)
+    dev = [torch.from_numpy(t).cuda().to(torch.bfloat16) for t in toks]
+    q, k, v, d_o = dev
+    hcfg = vd.HashCfg(B, w.N, w.L, w.k, 0, 0, 1)
+    keys, freqs, _ = vd.alloc_hash_outputs(hcfg)
+    hws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(hcfg))
+    vd.vardrop_hash(torch.from_numpy(x).cuda(), hcfg, keys, freqs, None, hws)
+    scfg = vd.SelectCfg(B, w.N, 0, w.rate, SEED, STEP)
+    sel = vd.alloc_select_outputs(scfg)
+    sws = vd.alloc_ws(vd.vardrop_select_workspace_bytes(scfg))
+    vd.vardrop_select(keys, scfg, sel["group_id"], sel["group_offsets"], sel["members"], sel["n_groups"], sel["sel_idx"], sel["n_sel"],
+                      sel["inv_idx"], sws)
+    acfg = vd.AttnCfg(B, w.N, w.H, w.D, 0.0, B)
+    aws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(acfg))
+    o = torch.zeros_like(q)
+    lse = torch.zeros((B, w.H, w.N), dtype=torch.float32, device="cuda")
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    vd.vardrop_attn_fwd(q, k, v, sel["sel_idx"], sel["n_sel"], acfg, o, lse, aws)
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, sel["sel_idx"], sel["n_sel"], sel["inv_idx"], acfg, dq, dk, dv, aws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(hws) == vd.OK and vd.ws_status(aws) == vd.OK
+    assert np.array_equal(keys.cpu().numpy().view(np.uint64), okeys)
+    want = oracle.select(okeys, 0, w.rate, SEED, STEP)
+    assert np.array_equal(sel["sel_idx"].cpu().numpy(), want["sel_idx"]) and np.array_equal(sel["n_sel"].cpu().numpy(), want["n_sel"])
+    assert len(set(want["n_sel"].tolist())) > 1 or not np.array_equal(want["sel_idx"][0], want["sel_idx"][1])
+    for b in (0, B - 1):
+        c = int(want["n_sel"][b]); idx = want["sel_idx"][b, :c]
+        cut = [t[b:b + 1].double().cpu().numpy() for t in dev]
+        wo, _ = oracle.attn_fwd(cut[0], cut[1], cut[2], idx)
+        assert_attn_close(o[b:b + 1, :c].double().cpu().numpy(), wo, f"o[{b}]")
+        wq, wk, wv = oracle.attn_bwd(cut[0], cut[1], cut[2], cut[3][:, :c], idx)
+        assert_attn_close(dq[b:b + 1].double().cpu().numpy(), wq, f"dq[{b}]")
+        assert_attn_close(dk[b:b + 1].double().cpu().numpy(), wk, f"dk[{b}]")
+        assert_attn_close(dv[b:b + 1].double().cpu().numpy(), wv, f"dv[{b}]")
