@@ -201,32 +201,45 @@ __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const Select
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kSmallMaxN = 2048;
 
-// Bitonic sort of M (a power of two) items in shared memory by M / 2 threads, one compare-exchange per thread and stage.
-// Items are (key, payload) pairs ordered by key, then payload.
-__device__ __forceinline__ void bitonic_sort_pairs(ulonglong2* a, int M) {
+// Bitonic sort of M (a power of two >= 64) items by M / 2 threads.  Thread t keeps items 2t and 2t + 1 in registers.
+// Compare-exchange distance j = 1 stays inside the thread, j = 2 .. 32 goes through warp shuffles (the partner of item
+// i is item i ^ j = slot (i & 1) of lane t ^ (j / 2)), and only j >= 64 passes through shared memory.
+// Items are (key, payload) pairs ordered by key, then payload; kPayload = false sorts bare keys.
+template <bool kPayload>
+__device__ __forceinline__ void bitonic_sort_regs(uint64_t& k0, uint32_t& p0, uint64_t& k1, uint32_t& p1, uint64_t* sk, uint32_t* sp, int M) {
     const int t = threadIdx.x;
+    auto greater = [](uint64_t ka, uint32_t pa, uint64_t kb, uint32_t pb) { return ka > kb || (kPayload && ka == kb && pa > pb); };
+    // keep the smaller of (mine, other) when `want_min`, else the larger
+    auto keep = [&](uint64_t& km, uint32_t& pm, uint64_t ko, uint32_t po, bool want_min) {
+        const bool mine_greater = greater(km, pm, ko, po);
+        if (mine_greater == want_min) { km = ko; pm = po; }
+    };
     for (int k = 2; k <= M; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // lower index of this thread's pair (bit j clear)
-            const int l = i | j;
-            const bool up = (i & k) == 0;
-            const ulonglong2 x = a[i], y = a[l];
-            const bool gt = x.x > y.x || (x.x == y.x && x.y > y.y);
-            if (gt == up) { a[i] = y; a[l] = x; }
+        const bool up = ((2 * t) & k) == 0;              // the same for both items of the thread once k >= 2
+        int j = k >> 1;
+        for (; j >= 64; j >>= 1) {                       // partners live in another warp
+            sk[2 * t] = k0; sk[2 * t + 1] = k1;
+            if (kPayload) { sp[2 * t] = p0; sp[2 * t + 1] = p1; }
             __syncthreads();
+            const int l = (2 * t) ^ j;
+            const uint64_t ok0 = sk[l], ok1 = sk[l + 1];
+            const uint32_t op0 = kPayload ? sp[l] : 0u, op1 = kPayload ? sp[l + 1] : 0u;
+            __syncthreads();
+            const bool lower = ((2 * t) & j) == 0;
+            keep(k0, p0, ok0, op0, lower == up);
+            keep(k1, p1, ok1, op1, lower == up);
         }
-    }
-}
-__device__ __forceinline__ void bitonic_sort_u64(uint64_t* a, int M) {
-    const int t = threadIdx.x;
-    for (int k = 2; k <= M; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-            const int l = i | j;
-            const bool up = (i & k) == 0;
-            const uint64_t x = a[i], y = a[l];
-            if ((x > y) == up) { a[i] = y; a[l] = x; }
-            __syncthreads();
+        for (; j >= 2; j >>= 1) {                        // partners live in the same warp
+            const int m = j >> 1;
+            const uint64_t ok0 = __shfl_xor_sync(0xffffffffu, k0, m), ok1 = __shfl_xor_sync(0xffffffffu, k1, m);
+            const uint32_t op0 = kPayload ? __shfl_xor_sync(0xffffffffu, p0, m) : 0u, op1 = kPayload ? __shfl_xor_sync(0xffffffffu, p1, m) : 0u;
+            const bool lower = (t & m) == 0;
+            keep(k0, p0, ok0, op0, lower == up);
+            keep(k1, p1, ok1, op1, lower == up);
+        }
+        if (greater(k0, p0, k1, p1) == up) {             // distance 1: the thread's own pair (up is taken at k >= 2; k = 2 sorts pairs
+            const uint64_t tk = k0; k0 = k1; k1 = tk;    //              alternately up and down by bit 1 of the item index)
+            const uint32_t tp = p0; p0 = p1; p1 = tp;
         }
     }
 }
@@ -257,8 +270,7 @@ __device__ __forceinline__ int block_scan_pair(int v0, int v1, int* warp_sums, i
 // launched with M / 2 threads (M >= 64 a power of two, N <= M)
 __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const SelectParams P, int M) {
     extern __shared__ __align__(16) unsigned char sm_raw[];
-    ulonglong2* a2 = reinterpret_cast<ulonglong2*>(sm_raw);       // [M] (key, variate) pairs
-    uint64_t* a = reinterpret_cast<uint64_t*>(a2 + M);            // [M] (group, priority, rank) codes
+    uint64_t* a = reinterpret_cast<uint64_t*>(sm_raw);            // [M] sorted keys, later sorted (group, priority, rank) codes
     uint32_t* idx = reinterpret_cast<uint32_t*>(a + M);           // [M] variate by sorted position
     int* gpos = reinterpret_cast<int*>(idx + M);                  // [M] group id by sorted position
     int* off_s = gpos + M;                                        // [M + 1] group offsets
@@ -271,58 +283,57 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
     int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
     int32_t* sel = P.sel_idx + static_cast<size_t>(s) * N;
     int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
-    const int p0 = 2 * tid, p1 = 2 * tid + 1;                     // the two positions this thread owns outside the sorts
+    const int p0 = 2 * tid, p1 = 2 * tid + 1;                     // the two items / positions this thread owns
 
     if (s == 0 && tid == 0) *P.status = VARDROP_OK;               // nothing in this kernel can fail on the device
-    a2[p0] = make_ulonglong2(p0 < N ? keys[p0] : ~0ull, static_cast<uint64_t>(p0));
-    a2[p1] = make_ulonglong2(p1 < N ? keys[p1] : ~0ull, static_cast<uint64_t>(p1));
+    uint64_t k0 = p0 < N ? keys[p0] : ~0ull, k1 = p1 < N ? keys[p1] : ~0ull;
+    uint32_t n0 = p0, n1 = p1;
+    bitonic_sort_regs<true>(k0, n0, k1, n1, a, idx, M);
+    a[p0] = k0; a[p1] = k1; idx[p0] = n0; idx[p1] = n1;
     __syncthreads();
-    bitonic_sort_pairs(a2, M);
 
     // group heads -> dense ids and offsets
-    const int h0 = (p0 < N) && (p0 == 0 || a2[p0].x != a2[p0 - 1].x);
-    const int h1 = (p1 < N) && (a2[p1].x != a2[p1 - 1].x);
+    const int h0 = (p0 < N) && (p0 == 0 || k0 != a[p0 - 1]);
+    const int h1 = (p1 < N) && (k1 != k0);
     int G = 0;
     const int before = block_scan_pair(h0, h1, warp_sums, &G);
+    const int g0 = before + h0 - 1, g1 = before + h0 + h1 - 1;
     if (p0 < N) {
-        const int g = before + h0 - 1, n = static_cast<int>(a2[p0].y);
-        gpos[p0] = g; idx[p0] = n;
-        if (h0) { off_s[g] = p0; off[g] = p0; }
-        members[p0] = n;
-        gid[n] = g;
+        gpos[p0] = g0;
+        if (h0) { off_s[g0] = p0; off[g0] = p0; }
+        members[p0] = n0;
+        gid[n0] = g0;
     }
     if (p1 < N) {
-        const int g = before + h0 + h1 - 1, n = static_cast<int>(a2[p1].y);
-        gpos[p1] = g; idx[p1] = n;
-        if (h1) { off_s[g] = p1; off[g] = p1; }
-        members[p1] = n;
-        gid[n] = g;
+        gpos[p1] = g1;
+        if (h1) { off_s[g1] = p1; off[g1] = p1; }
+        members[p1] = n1;
+        gid[n1] = g1;
     }
     if (tid == 0) { off_s[G] = N; P.n_groups[s] = G; }
     for (int i = G + tid; i <= N; i += blockDim.x) off[i] = N;
     __syncthreads();
 
     // sampling rank: sort (group, priority, j)
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-        const int p = 2 * tid + e;
-        uint64_t c = ~0ull;
-        if (p < N) {
-            const int g = gpos[p];
-            const int j = p - off_s[g];
-            const uint32_t pri = philox4x32_10_word0(static_cast<uint32_t>(j), static_cast<uint32_t>(g), static_cast<uint32_t>(s), P.step,
-                                                     P.seed_lo, P.seed_hi);
-            c = (static_cast<uint64_t>(g) << 43) | (static_cast<uint64_t>(pri) << 11) | static_cast<uint64_t>(j);
-        }
-        a[p] = c;
+    uint64_t c0 = ~0ull, c1 = ~0ull;
+    if (p0 < N) {
+        const int j = p0 - off_s[g0];
+        const uint32_t pri = philox4x32_10_word0(static_cast<uint32_t>(j), static_cast<uint32_t>(g0), static_cast<uint32_t>(s), P.step, P.seed_lo, P.seed_hi);
+        c0 = (static_cast<uint64_t>(g0) << 43) | (static_cast<uint64_t>(pri) << 11) | static_cast<uint64_t>(j);
     }
-    __syncthreads();
-    bitonic_sort_u64(a, M);
+    if (p1 < N) {
+        const int j = p1 - off_s[g1];
+        const uint32_t pri = philox4x32_10_word0(static_cast<uint32_t>(j), static_cast<uint32_t>(g1), static_cast<uint32_t>(s), P.step, P.seed_lo, P.seed_hi);
+        c1 = (static_cast<uint64_t>(g1) << 43) | (static_cast<uint64_t>(pri) << 11) | static_cast<uint64_t>(j);
+    }
+    uint32_t d0 = 0, d1 = 0;
+    __syncthreads();                                              // everyone is done reading the sorted keys in `a`
+    bitonic_sort_regs<false>(c0, d0, c1, d1, a, nullptr, M);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
         const int q = 2 * tid + e;
+        const uint64_t c = e ? c1 : c0;
         if (q < N) {
-            const uint64_t c = a[q];
             const int g = static_cast<int>(c >> 43), j = static_cast<int>(c & 2047u);
             const int begin = off_s[g], size = off_s[g + 1] - begin;
             keep_s[idx[begin + j]] = (q - begin) < quota_of(size, P.gs, P.rate_ppm);
@@ -331,11 +342,11 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
     __syncthreads();
 
     // compaction in ascending variate order
-    const int k0 = p0 < N ? keep_s[p0] : 0, k1 = p1 < N ? keep_s[p1] : 0;
+    const int kp0 = p0 < N ? keep_s[p0] : 0, kp1 = p1 < N ? keep_s[p1] : 0;
     int total = 0;
-    int pos = block_scan_pair(k0, k1, warp_sums, &total);
-    if (p0 < N) { if (k0) { sel[pos] = p0; inv[p0] = pos; ++pos; } else inv[p0] = -1; }
-    if (p1 < N) { if (k1) { sel[pos] = p1; inv[p1] = pos; } else inv[p1] = -1; }
+    int pos = block_scan_pair(kp0, kp1, warp_sums, &total);
+    if (p0 < N) { if (kp0) { sel[pos] = p0; inv[p0] = pos; ++pos; } else inv[p0] = -1; }
+    if (p1 < N) { if (kp1) { sel[pos] = p1; inv[p1] = pos; } else inv[p1] = -1; }
     for (int i = total + tid; i < N; i += blockDim.x) sel[i] = -1;
     if (tid == 0) P.n_sel[s] = total;
 }
@@ -391,7 +402,7 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
     if (c.N <= kSmallMaxN) {
         int M = 64;
         while (M < c.N) M <<= 1;
-        const size_t smem = static_cast<size_t>(M) * (16 + 8 + 4 + 4 + 4 + 4) + 16;
+        const size_t smem = static_cast<size_t>(M) * (8 + 4 + 4 + 4 + 4) + 16;
         static thread_local int attr_dev = -1;
         int dev = 0;
         cudaGetDevice(&dev);
