@@ -221,8 +221,8 @@ def kernel_work(w, n_sel):
         "gather_kernel": ("hbm", 2 * 3 * kept * row),
         "attn_fwd_kernel": ("tensor", 4.0 * w.B * w.H * n_sel * n_sel * w.D),
         "bwd_prep_kernel": ("hbm", 2 * kept * row + kept * row + kept * w.H * 64 * 4),
-        "attn_bwd_kernel": ("tensor", 10.0 * w.B * w.H * n_sel * n_sel * w.D),
-        "bwd_finish_kernel": ("hbm", 3 * w.B * w.N * row + kept * w.H * 64 * 4),
+        "attn_bwd_kernel": ("tensor", 10.0 * w.B * w.H * n_sel * n_sel * w.D),      # also writes the zero rows of the dropped variates
+        "bwd_convert_kernel": ("hbm", kept * row + kept * w.H * 64 * 4),
     }
 
 

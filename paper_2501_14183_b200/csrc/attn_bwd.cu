@@ -7,8 +7,10 @@
 //                    row of tensor memory; P^T and dS^T are written to shared memory once and feed three
 //                    tensor-core products: dV += P^T dO, dK += dS^T Q (accumulated in tensor memory across the
 //                    query loop) and dQ_i = dS K (added into the fp32 accumulator with atomics).
-// bwd_finish_kernel  dq rows from the accumulator (scaled, bf16) and zero rows for every dropped variate, so
-//                    each row of dq / dk / dv is written exactly once.
+//                    The same kernel writes the zero rows of every dropped variate (while its first tiles are in
+//                    flight) and, when the CTA that finishes the last key tile of an (instance, head) pair sees the
+//                    pair complete, converts that pair's dQ' accumulator to bf16 rows of dq: each row of dq / dk / dv
+//                    is written exactly once and no further launch is needed.
 #include "attn_common.cuh"
 
 namespace vardrop {
@@ -85,6 +87,10 @@ struct BwdParams {
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     const int32_t* sel_idx; // [S, N]; NULL: identity
+    const int32_t* inv_idx; // [S, N]; NULL: identity (nothing dropped)
+    int32_t* tile_done;     // [B, H] key tiles finished per (instance, head); zeroed by the forward pass
+    int convert_here;       // 1: the CTA that completes an (instance, head) pair converts its dQ' accumulator to dq rows
+                            // 0: a separate kernel does (many tiles: the conversion wants the whole GPU)
     const int32_t* n_sel;   // [S]; NULL: N
     int* status;
     int B, N, Ncap, H, D, S;
@@ -123,6 +129,33 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     extern __shared__ unsigned char smem_dyn[];
     const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
+    if (P.inv_idx) {            // zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid
+        const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
+        const int total_rows = P.B * P.N;
+        const int lane = threadIdx.x & 31;
+        const int warps_grid = gridDim.x * (blockDim.x >> 5);
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
+        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
+        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
+        int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
+        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
+        for (int base = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
+            const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
+            bool dropped = false;
+            if (lane < group && r < total_rows) {
+                const int b = r / P.N, n = r - b * P.N;
+                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
+            }
+            unsigned mask = __ballot_sync(0xffffffffu, dropped);
+            while (mask) {
+                const int l = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
+                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
+            }
+        }
+    }
     if (static_cast<int>(blockIdx.x) >= n_items) return;
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
@@ -422,6 +455,29 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             tc_fence_before();
             __syncthreads();        // the accumulators are read out before the next item's products overwrite them
         }
+        if (P.convert_here && !single_tile && ok) {   // dQ' of this (instance, head) is complete once all its key tiles are: the last one converts it
+            int* flag = reinterpret_cast<int*>(smem_dyn + 60);
+            if (tid == 0) {
+                bulk_wait_group0();                      // this item's reductions have landed
+                __threadfence();
+                *flag = atomicAdd(P.tile_done + b * P.H + h, 1) == n_q - 1;
+            }
+            __syncthreads();
+            if (*flag) {
+                __threadfence();
+                const int chunks_head = P.D / 8;         // 16-byte output chunks per row
+                for (int idx = tid; idx < n_sel * chunks_head; idx += blockDim.x) {
+                    const int j = idx / chunks_head, dc = idx - j * chunks_head;
+                    const float4* acc = reinterpret_cast<const float4*>(P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * kDP) + dc * 2;
+                    const float4 a0 = __ldcg(acc), a1 = __ldcg(acc + 1);
+                    const int n = sel ? sel[j] : j;
+                    *reinterpret_cast<uint4*>(P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + dc * 8) =
+                        make_uint4(pack2(a0.x * P.scale, a0.y * P.scale), pack2(a0.z * P.scale, a0.w * P.scale),
+                                   pack2(a1.x * P.scale, a1.y * P.scale), pack2(a1.z * P.scale, a1.w * P.scale));
+                }
+            }
+            __syncthreads();        // `flag` is free for the next item
+        }
         ++n_done;
     }
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
@@ -432,22 +488,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// finish
+// dq from the accumulator (paths with many key tiles)
 // ---------------------------------------------------------------------------------------------------------
-struct FinishParams {
+struct ConvertParams {
     const float4* dq_acc;    // [B, Ncap, H, 64] fp32
-    uint4 *dq, *dk, *dv;     // [B, N, H, D] bf16
+    uint4* dq;               // [B, N, H, D] bf16
     const int32_t* inv_idx;  // [S, N]; NULL: identity
     const int32_t* n_sel;    // [S]; NULL: N
     int N, Ncap, H, D, S;
     float scale;
 };
 
-__global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
+__global__ void __launch_bounds__(256) bwd_convert_kernel(const ConvertParams P) {
     const int b = blockIdx.y;
     const int srow = P.S > 1 ? b : 0;
+    if ((P.n_sel ? P.n_sel[srow] : P.N) <= kTile) return;       // single key tile: the main kernel wrote the kept dq rows
     const int32_t* inv = P.inv_idx ? P.inv_idx + static_cast<size_t>(srow) * P.N : nullptr;
-    const bool dq_done = (P.n_sel ? P.n_sel[srow] : P.N) <= kTile;      // single key tile: the main kernel wrote the kept dq rows
     const int chunks_head = P.D / 8;
     const int chunks_row = P.H * chunks_head;
     const int total = P.N * chunks_row;
@@ -456,19 +512,11 @@ __global__ void __launch_bounds__(256) bwd_finish_kernel(const FinishParams P) {
         const int c = idx - n * chunks_row;
         const int h = c / chunks_head, dc = c - h * chunks_head;
         const int j = inv ? inv[n] : n;
-        const size_t dst = static_cast<size_t>(b) * total + idx;
-        if (j >= 0) {
-            if (dq_done) continue;
-            const float4* src = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * (kDP / 4) + dc * 2;
-            const float4 a = __ldcg(src), c2 = __ldcg(src + 1);
-            P.dq[dst] = make_uint4(pack2(a.x * P.scale, a.y * P.scale), pack2(a.z * P.scale, a.w * P.scale),
-                                   pack2(c2.x * P.scale, c2.y * P.scale), pack2(c2.z * P.scale, c2.w * P.scale));
-        } else {
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            P.dq[dst] = z;
-            P.dk[dst] = z;
-            P.dv[dst] = z;
-        }
+        if (j < 0) continue;                                     // dropped rows were zeroed by the main kernel
+        const float4* src = P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * (kDP / 4) + dc * 2;
+        const float4 a = __ldcg(src), c2 = __ldcg(src + 1);
+        P.dq[static_cast<size_t>(b) * total + idx] = make_uint4(pack2(a.x * P.scale, a.y * P.scale), pack2(a.z * P.scale, a.w * P.scale),
+                                                                pack2(c2.x * P.scale, c2.y * P.scale), pack2(c2.z * P.scale, c2.w * P.scale));
     }
 }
 
@@ -531,6 +579,9 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     P.src_do.idx = nullptr;         // dO rows are already compact: slot j is row j
     P.dq = static_cast<__nv_bfloat16*>(dq); P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
     P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
+    P.inv_idx = sel_idx ? inv_idx : nullptr;
+    P.tile_done = reinterpret_cast<int32_t*>(base + w.tile_done);
+    P.convert_here = gathered ? 1 : 0;
     P.status = reinterpret_cast<int*>(base);
     P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D; P.S = attn_sel_rows(c);
     P.scale = scale; P.scale_log2 = scale * 1.4426950408889634f;
@@ -548,21 +599,22 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         attn_bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, macc, P);
     }
     if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
-
-    FinishParams F{};
-    F.dq_acc = reinterpret_cast<const float4*>(base + w.dq_acc);
-    F.dq = static_cast<uint4*>(dq); F.dk = static_cast<uint4*>(dk); F.dv = static_cast<uint4*>(dv);
-    F.inv_idx = sel_idx ? inv_idx : nullptr;
-    F.n_sel = sel_idx ? n_sel : nullptr;
-    F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.S = attn_sel_rows(c); F.scale = scale;
-    {
+    if (!gathered && c.N > kTile) {         // several key tiles possible: dq comes from the accumulator in a pass of its own
+        ConvertParams F{};
+        F.dq_acc = reinterpret_cast<const float4*>(base + w.dq_acc);
+        F.dq = static_cast<uint4*>(dq);
+        F.inv_idx = sel_idx ? inv_idx : nullptr;
+        F.n_sel = sel_idx ? n_sel : nullptr;
+        F.N = c.N; F.Ncap = w.Ncap; F.H = c.H; F.D = c.D; F.S = attn_sel_rows(c); F.scale = scale;
         const long long work = static_cast<long long>(c.N) * c.H * (c.D / 8);
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 8 * sm_count() / c.B);
         if (gx > cap) gx = cap;
-        { LaunchScope ls_(K_BWD_FINISH, stream); bwd_finish_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F); }
+        { LaunchScope ls_(K_BWD_CONVERT, stream); bwd_convert_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F); }
+        if (int st = check_cuda(cudaGetLastError(), "attention: backward convert launch")) return st;
     }
-    return check_cuda(cudaGetLastError(), "attention: backward finish launch");
+    return VARDROP_OK;
+
 }
 
 }  // namespace vardrop

@@ -17,6 +17,7 @@ struct AttnWs {
     size_t qg, kg, vg, dog;   // staged [B, Ncap, H, 64] bf16 copies (gathered and/or padded)
     size_t delta;             // [B, H, Ncap] fp32
     size_t dq_acc;            // [B, Ncap, H, 64] fp32
+    size_t tile_done;         // [B, H] int32: key tiles of (b, h) whose backward work is complete
     size_t total;
     int Ncap;
 };
@@ -32,6 +33,7 @@ inline AttnWs attn_layout(const vardrop_attn_cfg& c) {
     w.dog = o; o += align_up(staged, 1024);
     w.delta = o; o += align_up(sizeof(float) * c.B * c.H * w.Ncap, 1024);
     w.dq_acc = o; o += align_up(staged * 2, 1024);
+    w.tile_done = o; o += align_up(sizeof(int32_t) * c.B * c.H, 1024);
     w.total = o;
     return w;
 }

@@ -140,6 +140,7 @@ struct FwdParams {
     const int32_t* n_sel;   // [S] kept counts; NULL: all N tokens
     int* status;
     float4* dq_acc;         // [B, Ncap, H, 64] fp32: zeroed here for the backward pass when it will accumulate into it
+    int32_t* tile_done;     // [B, H] completion counters of the backward pass, zeroed here
     TileSource src;         // where Q, K, V tiles come from
     int B, N, Ncap, H, D, S;
     float scale_log2;       // sm_scale * log2(e)
@@ -257,6 +258,7 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
             load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, src, 0, n_sel, h, b, P.H);
             load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, src, 0, n_sel, h, b, P.H);
         }
+        if (qt == 0 && tid == 0) P.tile_done[b * P.H + h] = 0;
         if (n_kv > 1) {             // the backward pass will add per-key-tile pieces of dQ' into the accumulator: clear this tile's rows
 #pragma unroll
             for (int x = 0; x < kDP / 4; ++x) {          // 16 consecutive threads clear one 256-byte row
@@ -419,6 +421,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
     P.o = static_cast<__nv_bfloat16*>(o); P.lse = lse; P.n_sel = sel_idx ? n_sel : nullptr;
     P.status = reinterpret_cast<int*>(base);
     P.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
+    P.tile_done = reinterpret_cast<int32_t*>(base + w.tile_done);
     P.src.idx = sel_idx; P.src.gathered = attn_uses_gather(c, sel_idx) ? 1 : 0; P.src.tokens = c.N;
     P.src.rows_total = c.B * c.N * c.H;
     P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D; P.S = attn_sel_rows(c);
