@@ -129,7 +129,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     extern __shared__ unsigned char smem_dyn[];
     const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
-    if (P.inv_idx) {            // zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid
+    // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
+    // operand loads of its first work item, so the stores drain while those loads are in flight.
+    bool zeros_written = P.inv_idx == nullptr;
+    auto write_zero_rows = [&]() {
+        zeros_written = true;
         const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
         const int total_rows = P.B * P.N;
         const int lane = threadIdx.x & 31;
@@ -155,8 +159,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
             }
         }
+    };
+    if (static_cast<int>(blockIdx.x) >= n_items) {
+        if (!zeros_written) write_zero_rows();
+        return;
     }
-    if (static_cast<int>(blockIdx.x) >= n_items) return;
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
     uint64_t* bar_kv = bars + 0;
@@ -292,6 +299,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         uint4 o_cur[4], o_next[4];
         float dl_cur = load_delta(b, h, row), dl_next = 0.f;
         if (!use_delta) load_o(b, h, row, o_cur);
+        if (!zeros_written) write_zero_rows();
         const int key = jt * kTile + row;               // this thread's key row
         const bool key_valid = key < n_sel;
 
@@ -480,6 +488,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
         ++n_done;
     }
+    if (!zeros_written) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
     tc_fence_before();
