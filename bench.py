@@ -331,7 +331,7 @@ def run_gpu(args):
                 "timing": "CUDA events around every launch, second pass of the same K steps",
                 "ms_per_step_with_timer_armed": ms_armed / args.steps}
 
-    cpu = cpu_baseline(w, reps=2)
+    cpu = None if args.no_cpu else cpu_baseline(w, reps=2)
     line = {
         "metric": METRIC, "value": dist_util.aggregate_throughput(w.tokens, world, ms / args.steps * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps,
@@ -446,6 +446,7 @@ def main():
     ap.add_argument("--workload", default="elec", choices=["tiny", "elec", "traffic", "long", "scale"])
     ap.add_argument("--impl", default="vardrop", choices=["vardrop", "reference"])
     ap.add_argument("--no-off", action="store_true", help="skip the VarDrop-off comparison pass")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline (profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -309,6 +309,10 @@ int hash_launch(const float* x, const vardrop_hash_cfg& c, uint64_t* keys, int32
                 cudaStream_t stream) {
     int f_lo, f_hi;
     if (int st = hash_validate(c, &f_lo, &f_hi)) return st;
+    {
+        const int st = hash_rows_launch(x, c, f_lo, f_hi, keys, freqs, amp_dbg, status, stream);
+        if (st >= 0) return st;
+    }
     HashParams P{};
     P.x = x; P.keys = keys; P.freqs = freqs; P.amp_dbg = amp_dbg; P.status = status;
     P.B = c.B; P.N = c.N; P.L = c.L; P.k = c.k; P.f_lo = f_lo; P.nf = f_hi - f_lo; P.scope = c.scope;

@@ -28,6 +28,11 @@ int hash_validate(const vardrop_hash_cfg& cfg, int* f_lo, int* f_hi);
 int hash_launch(const float* x, const vardrop_hash_cfg& cfg, uint64_t* keys, int32_t* freqs, float* amp_dbg, int* status,
                 cudaStream_t stream);
 
+// hash_rows.cu: register-blocked plans for selected lookback lengths; -1 = no plan for this configuration
+int hash_rows_launch(const float* x, const vardrop_hash_cfg& cfg, int f_lo, int f_hi, uint64_t* keys, int32_t* freqs, float* amp_dbg,
+                     int* status, cudaStream_t stream);
+int sm_count();       // multiprocessors of the current device
+
 // select.cu
 size_t select_workspace_bytes(const vardrop_select_cfg& cfg);
 int select_validate(const vardrop_select_cfg& cfg);
