@@ -20,7 +20,12 @@
  *     shape, short workspace, failed launch) are returned at once and nothing is launched.  Problems
  *     found on the device (non-finite amplitude, a bounded wait that ran out) are written to the
  *     first int32 of `ws` as a vardrop_status; read it with a device-to-host copy after
- *     synchronising the stream.  vardrop_last_error() gives a thread-local text for the last non-OK return.
+ *     synchronising the stream.  The word is sticky: the first device-side problem is recorded and stays
+ *     until the caller zeroes it, so zero the first int32 of a new workspace (and after handling an
+ *     error); the library itself never clears it, which keeps a problem of an earlier queued call
+ *     readable after later ones.  vardrop_last_error() gives a thread-local text for the last non-OK return.
+ *   - Kernels are launched with programmatic stream serialization: a kernel's set-up may overlap the
+ *     tail of the previous kernel on the same stream, its reads and writes do not.
  *   - Calls are thread-safe as long as concurrent calls use different workspaces.
  */
 #ifndef VARDROP_H_

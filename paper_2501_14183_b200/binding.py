@@ -159,7 +159,8 @@ def ws_status(ws) -> int:
 
 # ---- buffer helpers (allocation only) -----------------------------------------------------------------------
 def alloc_ws(nbytes: int, device="cuda"):
-    return torch.empty(max(256, (nbytes + 255) // 256 * 256), dtype=torch.uint8, device=device)
+    """A zero-filled workspace: its status word is only ever set by the library, never cleared."""
+    return torch.zeros(max(256, (nbytes + 255) // 256 * 256), dtype=torch.uint8, device=device)
 
 
 def alloc_hash_outputs(cfg: HashCfg, device="cuda", want_freqs=True, want_amp=False):

@@ -40,6 +40,8 @@ struct PrepParams {
 
 // one thread per 16-byte chunk of a staged (token, head) row; the 8 threads of a row reduce Delta by shuffles
 __global__ void __launch_bounds__(256) bwd_prep_kernel(const PrepParams P) {
+    chain_wait();
+    chain_release();
     const int b = blockIdx.y;
     const int n_sel = P.n_sel ? P.n_sel[P.S > 1 ? b : 0] : P.N;
     if (!P.dog && n_sel <= kTile) return;            // a single key tile: the main kernel computes Delta itself
@@ -127,7 +129,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                                                    const __grid_constant__ CUtensorMap map_do,
                                                                    const __grid_constant__ CUtensorMap map_acc, const BwdParams P) {
     extern __shared__ unsigned char smem_dyn[];
-    const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) + kTile - 1) / kTile;     // tiles of the longest selection
+    chain_wait();
+    chain_release();
+    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
+    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
     // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
     // operand loads of its first work item, so the stores drain while those loads are in flight.
@@ -275,7 +281,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int h = (item / n_t_max) % P.H;
         const int b = item / (n_t_max * P.H);
         const int srow = P.S > 1 ? b : 0;
-        n_sel = P.n_sel ? P.n_sel[srow] : P.N;
+        n_sel = P.S > 1 ? P.n_sel[srow] : kept_shared;
         const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
         if (jt >= n_q) continue;
         const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
@@ -283,25 +289,30 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
         TileSource src = P.src, src_do = P.src_do;
         if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
-        if (warp == 0) {            // every MMA of the previous item has completed: K, V and both Q/dO stages are free
+        // plain loads first (row statistics, forward output, the variate this thread's key row scatters to): they are in
+        // flight while the tile fetches are issued
+        const int key = jt * kTile + row;               // this thread's key row
+        const bool key_valid = key < n_sel;
+        const float lse_first = load_lse(b, h, row);
+        uint4 o_cur[4], o_next[4];
+        float dl_cur = load_delta(b, h, row), dl_next = 0.f;
+        if (!use_delta) load_o(b, h, row, o_cur);
+        const int n_out = key_valid ? (sel ? sel[key] : key) : 0;
+        {   // every MMA of the previous item has completed: K, V and both Q/dO stages are free.  Warps 0 .. 3 fetch K, V, Q, dO side
+            // by side (each looks up its own gather rows); the byte counts are announced by thread 0, and a barrier phase
+            // cannot complete before that arrival, whichever comes first.
             const uint32_t st0 = q_count & 1;
             if (tid == 0) {
                 mbar_expect_tx(bar_kv, 2 * kTileBytes);
                 mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
             }
-            __syncwarp();
-            load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, src, 0, n_sel, h, b, P.H);
-            load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, src_do, 0, n_sel, h, b, P.H);
+            if (warp == 0) load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            else if (warp == 1) load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            else if (warp == 2) load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, src, 0, n_sel, h, b, P.H);
+            else if (warp == 3) load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, src_do, 0, n_sel, h, b, P.H);
         }
-        if (half == 0) s_stat[(q_count & 1) * kTile + row] = load_lse(b, h, row);
-        uint4 o_cur[4], o_next[4];
-        float dl_cur = load_delta(b, h, row), dl_next = 0.f;
-        if (!use_delta) load_o(b, h, row, o_cur);
+        if (half == 0) s_stat[(q_count & 1) * kTile + row] = lse_first;
         if (!zeros_written) write_zero_rows();
-        const int key = jt * kTile + row;               // this thread's key row
-        const bool key_valid = key < n_sel;
 
         for (int i = 0; i < n_q; ++i, ++q_count) {
             const uint32_t st = q_count & 1, ph = q_count & 1;
@@ -331,11 +342,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             __syncthreads();                             // row statistics of this stage visible
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
-            if (warp == 0 && i + 1 < n_q) {              // scores of this tile done => every product of the previous tile is done:
+            if (i + 1 < n_q) {                           // scores of this tile done => every product of the previous tile is done:
                 if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);      // the other Q / dO stage is free
-                __syncwarp();
-                load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), src, (i + 1) * kTile, n_sel, h, b, P.H);
-                load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), src_do, (i + 1) * kTile, n_sel, h, b, P.H);
+                if (warp == 2) load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), src, (i + 1) * kTile, n_sel, h, b, P.H);
+                else if (warp == 3) load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), src_do, (i + 1) * kTile, n_sel, h, b, P.H);
             }
 
             // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
@@ -439,8 +449,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         tc_fence_after();
         {   // dV, dK of this key tile: every thread takes part in the warp-collective loads, only valid key rows store
             const bool store = ok && key_valid && half * 32 < P.D;
-            const int n = store ? (sel ? sel[key] : key) : 0;
-            const size_t out = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
+            const size_t out = ((static_cast<size_t>(b) * P.N + n_out) * P.H + h) * P.D + half * 32;
             float acc[32];
             tmem_ld32(tm_dv + lane_sel + half * 32, acc);
             tmem_ld_wait();
@@ -509,6 +518,8 @@ struct ConvertParams {
 };
 
 __global__ void __launch_bounds__(256) bwd_convert_kernel(const ConvertParams P) {
+    chain_wait();
+    chain_release();
     const int b = blockIdx.y;
     const int srow = P.S > 1 ? b : 0;
     if ((P.n_sel ? P.n_sel[srow] : P.N) <= kTile) return;       // single key tile: the main kernel wrote the kept dq rows
@@ -556,8 +567,9 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 4 * sm_count() / c.B);              // about four CTAs per SM in total
         if (gx > cap) gx = cap;
-        { LaunchScope ls_(K_BWD_PREP, stream); bwd_prep_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(R); }
-        if (int st = check_cuda(cudaGetLastError(), "attention: backward prep launch")) return st;
+        cudaError_t perr;
+        { LaunchScope ls_(K_BWD_PREP, stream); perr = launch_chained(bwd_prep_kernel, dim3(gx, c.B), dim3(256), 0, stream, R); }
+        if (int st = check_cuda(perr, "attention: backward prep launch")) return st;
     }
 
     CUtensorMap mq, mk, mv, mdo;
@@ -605,9 +617,9 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
         const int grid = static_cast<int>(worst < sm_count() ? worst : sm_count());      // one CTA per SM (all of tensor memory)
         LaunchScope ls_(K_ATTN_BWD, stream);
-        attn_bwd_kernel<<<grid, kBwdThreads, kBwdSmemBytes, stream>>>(mq, mk, mv, mdo, macc, P);
+        const cudaError_t err = launch_chained(attn_bwd_kernel, dim3(grid), dim3(kBwdThreads), kBwdSmemBytes, stream, mq, mk, mv, mdo, macc, P);
+        if (int st = check_cuda(err, "attention: backward launch")) return st;
     }
-    if (int st = check_cuda(cudaGetLastError(), "attention: backward launch")) return st;
     if (!gathered && c.N > kTile) {         // several key tiles possible: dq comes from the accumulator in a pass of its own
         ConvertParams F{};
         F.dq_acc = reinterpret_cast<const float4*>(base + w.dq_acc);
@@ -619,8 +631,9 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 8 * sm_count() / c.B);
         if (gx > cap) gx = cap;
-        { LaunchScope ls_(K_BWD_CONVERT, stream); bwd_convert_kernel<<<dim3(gx, c.B), 256, 0, stream>>>(F); }
-        if (int st = check_cuda(cudaGetLastError(), "attention: backward convert launch")) return st;
+        cudaError_t cerr;
+        { LaunchScope ls_(K_BWD_CONVERT, stream); cerr = launch_chained(bwd_convert_kernel, dim3(gx, c.B), dim3(256), 0, stream, F); }
+        if (int st = check_cuda(cerr, "attention: backward convert launch")) return st;
     }
     return VARDROP_OK;
 

@@ -70,22 +70,37 @@ struct TileSource {
     int tokens;            // tokens per instance in the gathered tensor
     int rows_total;        // B * tokens * H
 };
-__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* map, uint64_t* bar, const TileSource& src, int tok0, int n_valid,
-                                          int h, int b, int H) {
+// Rows of the [rows, 64] view that the four slots tok0 + 4 lane .. + 3 of a gathered tile name (a row past the end for
+// slots at or past n_valid).  `picks` are the four entries idx[tok0 + 4 lane ..] (see tile_picks), fetched ahead of
+// time so that several tiles over the same slots share one fetch.
+__device__ __forceinline__ int4 tile_picks(const TileSource& src, int tok0) {
+    const int lane = threadIdx.x & 31;
+    const int slot = tok0 + 4 * lane;
+    if (!src.gathered || !src.idx) return make_int4(slot, slot + 1, slot + 2, slot + 3);
+    int4 p;
+    p.x = slot + 0 < src.tokens ? src.idx[slot + 0] : -1;
+    p.y = slot + 1 < src.tokens ? src.idx[slot + 1] : -1;
+    p.z = slot + 2 < src.tokens ? src.idx[slot + 2] : -1;
+    p.w = slot + 3 < src.tokens ? src.idx[slot + 3] : -1;
+    return p;
+}
+__device__ __forceinline__ void load_tile_picked(unsigned char* dst, const CUtensorMap* map, uint64_t* bar, const TileSource& src, int4 picks,
+                                                 int tok0, int n_valid, int h, int b, int H) {
     const int lane = threadIdx.x & 31;
     if (!src.gathered) {
         if (lane == 0) tma_load_4d(dst, map, bar, 0, h, tok0, b);
         return;
     }
+    const int slot = tok0 + 4 * lane;
+    const int n[4] = {picks.x, picks.y, picks.z, picks.w};
     int rows[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int slot = tok0 + 4 * lane + e;
-        int n = -1;
-        if (slot < n_valid) n = src.idx ? src.idx[slot] : slot;
-        rows[e] = n >= 0 ? (b * src.tokens + n) * H + h : src.rows_total;
-    }
+    for (int e = 0; e < 4; ++e) rows[e] = (slot + e < n_valid && n[e] >= 0) ? (b * src.tokens + n[e]) * H + h : src.rows_total;
     tma_gather4(dst + lane * 4 * kRowBytes, map, bar, 0, rows[0], rows[1], rows[2], rows[3]);
+}
+__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* map, uint64_t* bar, const TileSource& src, int tok0, int n_valid,
+                                          int h, int b, int H) {
+    load_tile_picked(dst, map, bar, src, tile_picks(src, tok0), tok0, n_valid, h, b, H);
 }
 
 // Three ways for the operand tiles to reach shared memory:

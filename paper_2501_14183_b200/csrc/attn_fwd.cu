@@ -110,6 +110,8 @@ struct GatherParams {
 };
 
 __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
+    chain_wait();
+    chain_release();
     const int b = blockIdx.y, t = blockIdx.z;
     const int srow = P.S > 1 ? b : 0;                                         // selection row of this instance
     const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
@@ -179,7 +181,11 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                                                                 const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v, const FwdParams P) {
     extern __shared__ unsigned char smem_dyn[];
-    const int n_t_max = (max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) + kTile - 1) / kTile;     // tiles of the longest selection
+    chain_wait();
+    chain_release();
+    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
+    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (query tile, head, instance); short instances skip tiles
     if (static_cast<int>(blockIdx.x) >= n_items) return;
 
@@ -242,21 +248,22 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
         const int h = (item / n_t_max) % P.H;
         const int b = item / (n_t_max * P.H);
         const int srow = P.S > 1 ? b : 0;
-        const int n_sel = P.n_sel ? P.n_sel[srow] : P.N;       // kept tokens of this instance
+        const int n_sel = P.S > 1 ? P.n_sel[srow] : kept_shared;       // kept tokens of this instance
         const int n_kv = (n_sel + kTile - 1) / kTile;          // its key tiles = query tiles
         if (qt >= n_kv) continue;
         TileSource src = P.src;
         if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
-        if (warp == 0) {            // every MMA of the previous item has completed: Q and both ring stages are free
+        {   // every MMA of the previous item has completed: Q and both ring stages are free.  Warps 0, 1, 2 fetch Q, K, V side
+            // by side (each looks up its own gather rows); the byte counts are announced by thread 0, and a barrier phase
+            // cannot complete before that arrival, whichever comes first.
             const uint32_t st0 = kv_count & 1;
             if (tid == 0) {
                 mbar_expect_tx(bar_q, kTileBytes);
                 mbar_expect_tx(bar_kv + st0, 2 * kTileBytes);
             }
-            __syncwarp();
-            load_tile(sQ, &map_q, bar_q, src, qt * kTile, n_sel, h, b, P.H);
-            load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, src, 0, n_sel, h, b, P.H);
-            load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, src, 0, n_sel, h, b, P.H);
+            if (warp == 0) load_tile(sQ, &map_q, bar_q, src, qt * kTile, n_sel, h, b, P.H);
+            else if (warp == 1) load_tile(sK + st0 * kTileBytes, &map_k, bar_kv + st0, src, 0, n_sel, h, b, P.H);
+            else if (warp == 2) load_tile(sV + st0 * kTileBytes, &map_v, bar_kv + st0, src, 0, n_sel, h, b, P.H);
         }
         if (qt == 0 && tid == 0) P.tile_done[b * P.H + h] = 0;
         if (n_kv > 1) {             // the backward pass will add per-key-tile pieces of dQ' into the accumulator: clear this tile's rows
@@ -275,11 +282,10 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
         for (int j = 0; j < n_kv; ++j, ++kv_count) {
             const uint32_t st = kv_count & 1;
             const uint32_t ph = kv_count & 1;            // bar_s / bar_o complete once per key tile
-            if (warp == 0 && j + 1 < n_kv) {             // the other stage was released by the wait on bar_o of the previous tile
+            if (j + 1 < n_kv) {                          // the other stage was released by the wait on bar_o of the previous tile
                 if (tid == 0) mbar_expect_tx(bar_kv + (st ^ 1), 2 * kTileBytes);
-                __syncwarp();
-                load_tile(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
-                load_tile(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
+                if (warp == 1) load_tile(sK + (st ^ 1) * kTileBytes, &map_k, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
+                else if (warp == 2) load_tile(sV + (st ^ 1) * kTileBytes, &map_v, bar_kv + (st ^ 1), src, (j + 1) * kTile, n_sel, h, b, P.H);
             }
             if (tid == 0) {
                 if (j == 0) {                            // later tiles: issued right behind the previous tile's P V
@@ -388,7 +394,6 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
                     const vardrop_attn_cfg& c, void* o, float* lse, void* ws, cudaStream_t stream) {
     const AttnWs w = attn_layout(c);
     char* base = static_cast<char*>(ws);
-    if (int st = check_cuda(cudaMemsetAsync(ws, 0, sizeof(int), stream), "attention: clear status")) return st;
     const bool staged = attn_uses_staging(c, sel_idx);
     CUtensorMap mq, mk, mv;
     if (staged) {
@@ -402,8 +407,9 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 4 * sm_count() / (3 * c.B));        // about four CTAs per SM in total; each strides over its rows
         if (gx > cap) gx = cap;
-        { LaunchScope ls_(K_GATHER, stream); gather_kernel<<<dim3(gx, c.B, 3), 256, 0, stream>>>(G); }
-        if (int st = check_cuda(cudaGetLastError(), "attention: gather launch")) return st;
+        cudaError_t gerr;
+        { LaunchScope ls_(K_GATHER, stream); gerr = launch_chained(gather_kernel, dim3(gx, c.B, 3), dim3(256), 0, stream, G); }
+        if (int st = check_cuda(gerr, "attention: gather launch")) return st;
         if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
         if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
@@ -434,13 +440,14 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         if (int st = check_cuda(cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFwdSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
+    cudaError_t err;
     {
         const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
         const int grid = static_cast<int>(worst < 2ll * sm_count() ? worst : 2ll * sm_count());      // two CTAs fit per SM
         LaunchScope ls_(K_ATTN_FWD, stream);
-        attn_fwd_kernel<<<grid, kFwdThreads, kFwdSmemBytes, stream>>>(mq, mk, mv, P);
+        err = launch_chained(attn_fwd_kernel, dim3(grid), dim3(kFwdThreads), kFwdSmemBytes, stream, mq, mk, mv, P);
     }
-    return check_cuda(cudaGetLastError(), "attention: forward launch");
+    return check_cuda(err, "attention: forward launch");
 }
 
 }  // namespace vardrop

@@ -37,6 +37,29 @@ __device__ __forceinline__ uint32_t fd_div(uint32_t t, FastDiv f) { return f.d =
 // device-side status: first error wins
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization: its CTAs may become resident and
+// run their set-up (shared-memory tables, barriers, tensor-memory allocation) while the previous kernel of the
+// stream is still finishing.  chain_wait() returns once that kernel has completed and its writes are visible: nothing
+// that another kernel produces or reads is touched before it.  chain_release() lets the next kernel's CTAs in.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- shared-memory addresses, mbarriers ------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 

@@ -188,6 +188,8 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
         sincospif(2.f * static_cast<float>(mf) / static_cast<float>(L), &s, &c);
         tw[m] = make_float2(c, -s);
     }
+    chain_wait();
+    chain_release();
     const int row0 = blockIdx.x * P.rows_per_cta;
     const int rows = min(P.rows_per_cta, P.rows_total - row0);
     for (int i = threadIdx.x; i < rows * nf; i += blockDim.x) acc[i] = 0.f;
@@ -361,8 +363,9 @@ int hash_launch(const float* x, const vardrop_hash_cfg& c, uint64_t* keys, int32
         attr_done_dev = dev;
     }
     const int grid = (P.rows_total + P.rows_per_cta - 1) / P.rows_per_cta;
-    { LaunchScope ls_(K_HASH, stream); hash_kernel<<<grid, kHashThreads, smem, stream>>>(P); }
-    return check_cuda(cudaGetLastError(), "hash: launch");
+    cudaError_t err;
+    { LaunchScope ls_(K_HASH, stream); err = launch_chained(hash_kernel, dim3(grid), dim3(kHashThreads), smem, stream, P); }
+    return check_cuda(err, "hash: launch");
 }
 
 }  // namespace vardrop

@@ -236,6 +236,8 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
         tw[m] = make_float2(c, -s);
     }
     __syncthreads();
+    chain_wait();
+    chain_release();
 
     const int rows_per_cta = kRowsWarps / P.team;
     const int member = warp % P.team;
@@ -395,8 +397,9 @@ int launch_rows(const RowsParams& P, cudaStream_t stream) {
     if (per_sm < 1) per_sm = 1;
     const int cap = sm_count() * per_sm;
     const int grid = want < cap ? want : cap;
-    { LaunchScope ls_(K_HASH, stream); hash_rows_kernel<L, R1, R2, PC, MINB><<<grid, kRowsThreads, smem, stream>>>(P); }
-    return check_cuda(cudaGetLastError(), "hash: launch");
+    cudaError_t err;
+    { LaunchScope ls_(K_HASH, stream); err = launch_chained(hash_rows_kernel<L, R1, R2, PC, MINB>, dim3(grid), dim3(kRowsThreads), smem, stream, P); }
+    return check_cuda(err, "hash: launch");
 }
 
 }  // namespace

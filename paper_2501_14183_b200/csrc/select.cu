@@ -102,6 +102,8 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectP
     __shared__ uint64_t skeys[kKeyChunk];
     __shared__ int warp_sums[kSelThreads / 32];
     __shared__ int flag;
+    chain_wait();
+    chain_release();
     const int s = blockIdx.z, N = P.N;
     const uint64_t* keys = P.keys + static_cast<size_t>(s) * N;
     int32_t* lt = P.lt + static_cast<size_t>(s) * N;
@@ -156,6 +158,8 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectP
 __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const SelectParams P) {
     __shared__ int warp_sums[kSelThreads / 32];
     __shared__ int flag;
+    chain_wait();
+    chain_release();
     const int s = blockIdx.z, N = P.N;
     const int32_t* members = P.members + static_cast<size_t>(s) * N;
     const int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
@@ -276,6 +280,8 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
     int* off_s = gpos + M;                                        // [M + 1] group offsets
     int* keep_s = off_s + M + 1;                                  // [M] kept flag by variate
     __shared__ int warp_sums[kSmallMaxN / 64];
+    chain_wait();
+    chain_release();
     const int s = blockIdx.x, N = P.N, tid = threadIdx.x;
     const uint64_t* keys = P.keys + static_cast<size_t>(s) * N;
     int32_t* members = P.members + static_cast<size_t>(s) * N;
@@ -410,16 +416,18 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
             if (int st = check_cuda(cudaFuncSetAttribute(select_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024), "select: smem attribute")) return st;
             attr_dev = dev;
         }
-        { LaunchScope ls_(K_SELECT_SMALL, stream); select_small_kernel<<<c.S, M / 2, smem, stream>>>(P, M); }
-        return check_cuda(cudaGetLastError(), "select: launch");
+        cudaError_t err;
+        { LaunchScope ls_(K_SELECT_SMALL, stream); err = launch_chained(select_small_kernel, dim3(c.S), dim3(M / 2), smem, stream, P, M); }
+        return check_cuda(err, "select: launch");
     }
     if (int st = check_cuda(cudaMemsetAsync(base, 0, w.zero_begin + w.zero_bytes, stream), "select: clear counters")) return st;
     const dim3 grid1((c.N + kSelThreads - 1) / kSelThreads, (c.N + kKeyChunk - 1) / kKeyChunk, c.S);
-    { LaunchScope ls_(K_SELECT_COUNT, stream); select_count_kernel<<<grid1, kSelThreads, 0, stream>>>(P); }
-    if (int st = check_cuda(cudaGetLastError(), "select: count launch")) return st;
+    cudaError_t err;
+    { LaunchScope ls_(K_SELECT_COUNT, stream); err = launch_chained(select_count_kernel, grid1, dim3(kSelThreads), 0, stream, P); }
+    if (int st = check_cuda(err, "select: count launch")) return st;
     const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
-    { LaunchScope ls_(K_SELECT_SAMPLE, stream); select_sample_kernel<<<grid2, kSelThreads, 0, stream>>>(P); }
-    return check_cuda(cudaGetLastError(), "select: sample launch");
+    { LaunchScope ls_(K_SELECT_SAMPLE, stream); err = launch_chained(select_sample_kernel, grid2, dim3(kSelThreads), 0, stream, P); }
+    return check_cuda(err, "select: sample launch");
 }
 
 // ---- allocation-free variant ------------------------------------------------------------------------------

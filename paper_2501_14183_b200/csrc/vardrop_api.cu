@@ -141,7 +141,6 @@ int vardrop_hash(const float* x, const vardrop_hash_cfg* cfg, uint64_t* keys, in
     VD_CHECK(check_ptr(amp_dbg, "amp_dbg", false));
     VD_CHECK(check_ws(ws, ws_bytes, hash_workspace_bytes(*cfg)));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    VD_CHECK(check_cuda(cudaMemsetAsync(ws, 0, sizeof(int), s), "hash: clear status"));
     return hash_launch(x, *cfg, keys, freqs, amp_dbg, static_cast<int*>(ws), s);
 }
 

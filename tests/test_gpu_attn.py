@@ -19,6 +19,7 @@ def run_attention(dev, B, N, H, D, sel, poison=True):
     ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
     if poison:
         ws.view(torch.int16).fill_(0x7FC1)        # bf16 NaN pattern everywhere in the scratch
+        ws[:4] = 0                                # except the status word, which the caller zeroes (the library only sets it)
     fill = float("nan") if poison else 0.0
     o = torch.full((B, N, H, D), fill, dtype=torch.bfloat16, device="cuda")
     lse = torch.full((B, H, N), fill, dtype=torch.float32, device="cuda")
@@ -128,6 +129,7 @@ def test_attention_per_instance_selections():
     cfg = vd.AttnCfg(B, N, H, D, 0.0, B)
     ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
     ws.view(torch.int16).fill_(0x7FC1)
+    ws[:4] = 0                                    # the status word is the caller's to zero
     nan = float("nan")
     o = torch.full((B, N, H, D), nan, dtype=torch.bfloat16, device="cuda")
     lse = torch.full((B, H, N), nan, dtype=torch.float32, device="cuda")
