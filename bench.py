@@ -209,37 +209,46 @@ def recorded_traffic(kernel, workload):
     return rec["dram_bytes_per_launch"]
 
 
-def kernel_work(w, n_sel):
-    """Algorithmic bytes / flops of one launch of each kernel (what the method must move or compute)."""
+def kernel_work(w, n_sel, selected=True):
+    """Algorithmic work of one launch of each kernel (what the method must move or compute): (bytes, flops).
+    flops is None for the kernels that only move data."""
     row = w.H * w.D * 2
     kept = w.B * n_sel
+    full = w.B * w.N
+    grads = 3 * (full if selected else kept) * row                  # dq, dk, dv come back in the full layout
     return {
-        "hash_kernel": ("hbm", w.B * w.N * w.L * 4 + w.N * (8 + 4 * w.k)),
-        "select_small_kernel": ("hbm", w.N * (8 + 6 * 4)),
-        "select_count_kernel": ("hbm", w.N * (8 + 4 * 4)),
-        "select_sample_kernel": ("hbm", w.N * 4 * 4),
-        "gather_kernel": ("hbm", 2 * 3 * kept * row),
-        "attn_fwd_kernel": ("tensor", 4.0 * w.B * w.H * n_sel * n_sel * w.D),
-        "bwd_prep_kernel": ("hbm", 2 * kept * row + kept * row + kept * w.H * 64 * 4),
-        "attn_bwd_kernel": ("tensor", 10.0 * w.B * w.H * n_sel * n_sel * w.D),      # also writes the zero rows of the dropped variates
-        "bwd_convert_kernel": ("hbm", kept * row + kept * w.H * 64 * 4),
+        "hash_kernel": (w.B * w.N * w.L * 4 + w.N * (8 + 4 * w.k), None),
+        "select_small_kernel": (w.N * (8 + 6 * 4), None),
+        "select_count_kernel": (w.N * (8 + 4 * 4), None),
+        "select_sample_kernel": (w.N * 4 * 4, None),
+        "gather_kernel": (2 * 3 * kept * row, None),
+        "attn_fwd_kernel": (3 * kept * row + kept * row + kept * w.H * 4, 4.0 * w.B * w.H * n_sel * n_sel * w.D),
+        "bwd_prep_kernel": (2 * kept * row + kept * row + kept * w.H * 64 * 4, None),
+        "attn_bwd_kernel": (5 * kept * row + kept * w.H * 4 + grads, 10.0 * w.B * w.H * n_sel * n_sel * w.D),
+        "bwd_convert_kernel": (kept * row + kept * w.H * 64 * 4, None),
     }
 
 
 def kernel_table(per_kernel, work, peaks):
+    """Per kernel: launches, average duration, share of the step, and the roofline that binds it.  A kernel with both
+    bytes and flops is bound by whichever needs longer at the measured peak (attention over a few hundred kept tokens
+    moves more bytes, relative to the HBM peak, than it computes relative to the tensor peak)."""
     kernels = {}
     total_ms = sum(v[0] for v in per_kernel.values()) or 1.0
     for name, (tot, n) in per_kernel.items():
         if n == 0:
             continue
-        bound, amount = work[name]
+        nbytes, flops = work[name]
         avg_s = tot / n * 1e-3
-        if bound == "hbm":
-            ach, peak, unit = amount / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
+        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+        t_tensor = flops / (peaks["bf16_tflops"] * 1e12) if flops else 0.0
+        if t_tensor > t_hbm:
+            bound, ach, peak, unit = "tensor", flops / avg_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
         else:
-            ach, peak, unit = amount / avg_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+            bound, ach, peak, unit = "hbm", nbytes / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
         kernels[name] = {"launches": n, "avg_us": tot / n * 1e3, "share": tot / total_ms, "bound": bound,
-                         "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak}
+                         "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                         "algorithmic_bytes": nbytes, "algorithmic_flops": flops}
     return kernels
 
 
@@ -311,7 +320,7 @@ def run_gpu(args):
         off = {"ms_per_step": ms_off / k_off, "tokens_per_s": w.tokens / (ms_off / k_off * 1e-3), "n_tokens": w.N,
                "attn_fwd_ms": pk_off["attn_fwd_kernel"][0] / k_off, "attn_bwd_ms": pk_off["attn_bwd_kernel"][0] / k_off,
                "attn_tflops": fl / t_attn / 1e12, "attn_frac_of_bf16_peak": fl / t_attn / 1e12 / peaks["bf16_tflops"],
-               "kernels": kernel_table(pk_off, kernel_work(w, w.N), peaks),
+               "kernels": kernel_table(pk_off, kernel_work(w, w.N, selected=False), peaks),
                "note": "timed with the per-kernel event timer armed"}
     clocks = sampler.stop() if rank == 0 else None
     path.check_status()

@@ -99,10 +99,27 @@ struct BwdParams {
     float scale, scale_log2;
 };
 
-constexpr int kBwdThreads = 256;       // two threads per tensor-memory lane: each takes one 64-column half
+constexpr int kBwdWorkers = 256;       // two threads per tensor-memory lane: each takes one 64-column half
+constexpr int kBwdThreads = kBwdWorkers + 32;   // plus one warp whose first lane issues every tensor-core product
 constexpr uint32_t kBwdTmemCols = 512;
-constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 4 * kTileBytes /*Q, dO x 2 stages*/ +
-                              4 * kTileBytes /*P^T, dS^T*/ + 2 * kTileBytes /*dQ tile, fp32, two 32-column halves*/;
+constexpr int kQStages = 3;            // ring of query-tile operands (Q and dO), fetched two tiles ahead
+constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 2 * kQStages * kTileBytes /*Q, dO ring*/ +
+                              4 * kTileBytes /*P^T, dS^T*/ + 2 * kTileBytes /*dQ tile, fp32, two 32-column halves*/;     // 227 KiB: all an SM offers a CTA
+
+// barrier among the worker threads only (the issuing warp never joins it)
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kBwdWorkers) : "memory"); }
+__device__ __forceinline__ bool worker_sync_and(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "bar.red.and.pred p, 1, %2, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(ok)), "n"(kBwdWorkers)
+        : "memory");
+    return r != 0;
+}
 
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
@@ -133,7 +150,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     chain_release();
     // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
-    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 56)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 88)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
     // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
     // operand loads of its first work item, so the stores drain while those loads are in flight.
@@ -143,14 +160,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
         const int total_rows = P.B * P.N;
         const int lane = threadIdx.x & 31;
-        const int warps_grid = gridDim.x * (blockDim.x >> 5);
+        const int warps_grid = gridDim.x * (kBwdWorkers >> 5);
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
         uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
         uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
         uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
         int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
         while (group < 32 && group * warps_grid < total_rows) group <<= 1;
-        for (int base = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
+        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
             const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
             bool dropped = false;
             if (lane < group && r < total_rows) {
@@ -167,24 +184,27 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
     };
     if (static_cast<int>(blockIdx.x) >= n_items) {
-        if (!zeros_written) write_zero_rows();
+        if (!zeros_written && threadIdx.x < kBwdWorkers) write_zero_rows();
         return;
     }
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
     uint64_t* bar_kv = bars + 0;
-    uint64_t* bar_qdo = bars + 1;                   // [2]
-    uint64_t* bar_s = bars + 3;
-    uint64_t* bar_g = bars + 4;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-    uint64_t* bar_acc = bars + 6;                   // every product of the item complete: dV, dK final, operands free
-    float* s_stat = reinterpret_cast<float*>(smem_dyn + 64);      // [2 stages][128] lse of the query tile, log2 domain
-    float* s_dpart = s_stat + 2 * kTile;                          // [2 halves][128] partial Delta = sum over 32 head dims of dO O
-    unsigned char* sK = align_tiles(smem_dyn + 64 + 4 * kTile * sizeof(float));
+    uint64_t* bar_qdo = bars + 1;                   // [3]
+    uint64_t* bar_s = bars + 4;                     // S^T of a query tile complete
+    uint64_t* bar_dp = bars + 5;                    // dP^T of a query tile complete (and every product issued before it)
+    uint64_t* bar_g = bars + 6;                     // dQ of a query tile complete
+    uint64_t* bar_acc = bars + 7;                   // every product of the item complete: dV, dK final, operands free
+    uint64_t* bar_p = bars + 8;                     // P^T of a query tile written by every worker thread
+    uint64_t* bar_ds = bars + 9;                    // dS^T of a query tile written by every worker thread
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 80);
+    float* s_stat = reinterpret_cast<float*>(smem_dyn + 128);     // [3 stages][128] lse of the query tile, log2 domain
+    float* s_dpart = s_stat + kQStages * kTile;                   // [2 halves][128] partial Delta = sum over 32 head dims of dO O
+    unsigned char* sK = align_tiles(smem_dyn + 128 + (kQStages + 2) * kTile * sizeof(float));
     unsigned char* sV = sK + kTileBytes;
-    unsigned char* sQ = sV + kTileBytes;            // 2 stages
-    unsigned char* sdO = sQ + 2 * kTileBytes;       // 2 stages
-    unsigned char* sPt = sdO + 2 * kTileBytes;      // P^T  : rows = keys, columns = queries (two 64-query panels)
+    unsigned char* sQ = sV + kTileBytes;            // 3 stages
+    unsigned char* sdO = sQ + kQStages * kTileBytes;   // 3 stages
+    unsigned char* sPt = sdO + kQStages * kTileBytes;  // P^T  : rows = keys, columns = queries (two 64-query panels)
     unsigned char* sdSt = sPt + 2 * kTileBytes;     // dS^T : same shape
     unsigned char* sDQ = sdSt + 2 * kTileBytes;     // dQ_i as fp32: panel `half` = head dimensions 32 half .. 32 half + 31, 128-byte swizzled rows
     if (sDQ + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
@@ -201,11 +221,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     }
     if (tid == 0) {
         mbar_init(bar_kv, 1);
-        mbar_init(bar_qdo + 0, 1);
-        mbar_init(bar_qdo + 1, 1);
+        for (int st = 0; st < kQStages; ++st) mbar_init(bar_qdo + st, 1);
         mbar_init(bar_s, 1);
+        mbar_init(bar_dp, 1);
         mbar_init(bar_g, 1);
         mbar_init(bar_acc, 1);
+        mbar_init(bar_p, kBwdWorkers);
+        mbar_init(bar_ds, kBwdWorkers);
         mbar_fence_init();
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_k);
@@ -231,7 +253,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     int n_sel = P.N;            // kept tokens of the instance being processed (set per work item)
     bool use_delta = false;     // precomputed Delta in use for this instance
     bool ok = true;
-    uint32_t q_count = 0;       // query tiles consumed so far by this CTA: stage = q_count & 1
+    uint32_t q_count = 0;       // query tiles consumed so far by this CTA: ring stage = q_count mod 3
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
 
     // operand descriptors, built once and stepped by additions: K-major views for the scores and the P^T / dS^T panels,
@@ -241,16 +263,41 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const uint64_t d_pt = umma_desc_sw128(smem_u32(sPt), 16, 1024), d_dst = umma_desc_sw128(smem_u32(sdSt), 16, 1024);
     const uint64_t m_q0 = umma_desc_sw128(smem_u32(sQ), kTileBytes, 1024), m_do0 = umma_desc_sw128(smem_u32(sdO), kTileBytes, 1024);
     const uint64_t m_dst = umma_desc_sw128(smem_u32(sdSt), kTileBytes, 1024), m_k = umma_desc_sw128(smem_u32(sK), kTileBytes, 1024);
-    // S^T = K Q^T and dP^T = V dO^T of the query tile in ring stage `stage` (issued by one thread), completion on bar_s
-    auto issue_scores = [&](uint32_t stage) {
-        const uint64_t dq_ = umma_desc_advance(d_q0, stage * kTileBytes), dd_ = umma_desc_advance(d_do0, stage * kTileBytes);
+    // The five products of a (key tile, query tile) pair, each issued by one thread.  S^T = K Q^T and dP^T = V dO^T read the
+    // query tile in ring stage `stage`; dV += P^T dO and dK += dS^T Q accumulate over the query loop; dQ_i = dS K.
+    auto issue_st = [&](uint32_t stage) {
+        const uint64_t dq_ = umma_desc_advance(d_q0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
             tc_mma_bf16(tm_st, umma_desc_advance(d_k, ks * 32), umma_desc_advance(dq_, ks * 32), idesc_kk, ks > 0);
+        tc_commit(bar_s);
+    };
+    auto issue_dpt = [&](uint32_t stage) {
+        const uint64_t dd_ = umma_desc_advance(d_do0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
             tc_mma_bf16(tm_dpt, umma_desc_advance(d_v, ks * 32), umma_desc_advance(dd_, ks * 32), idesc_kk, ks > 0);
-        tc_commit(bar_s);
+        tc_commit(bar_dp);
+    };
+    auto issue_dv = [&](uint32_t stage, uint32_t acc_on) {           // reduction over the 128 queries
+        const uint64_t mdo = umma_desc_advance(m_do0, stage * kTileBytes);
+#pragma unroll
+        for (int ks = 0; ks < kTile / 16; ++ks)
+            tc_mma_bf16(tm_dv, umma_desc_advance(d_pt, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mdo, ks * 2048), idesc_kmn,
+                        ks > 0 ? 1u : acc_on);
+    };
+    auto issue_dk = [&](uint32_t stage, uint32_t acc_on) {
+        const uint64_t mq = umma_desc_advance(m_q0, stage * kTileBytes);
+#pragma unroll
+        for (int ks = 0; ks < kTile / 16; ++ks)
+            tc_mma_bf16(tm_dk, umma_desc_advance(d_dst, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mq, ks * 2048), idesc_kmn,
+                        ks > 0 ? 1u : acc_on);
+    };
+    auto issue_dq = [&]() {                                           // reduction over the 128 keys
+#pragma unroll
+        for (int ks = 0; ks < kTile / 16; ++ks)
+            tc_mma_bf16(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
+        tc_commit(bar_g);
     };
 
     // lse of query `qrow` in the log2 domain (fetched by the threads of half 0; +inf switches a missing query off)
@@ -289,49 +336,129 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
         TileSource src = P.src, src_do = P.src_do;
         if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
+        if (warp == kBwdWorkers / 32) {
+            // The issuing warp: its first lane queues the products as their operands become ready.  The workers announce
+            // P^T and dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and
+            // the next dP^T while they compute the next P^T.
+            if ((tid & 31) == 0) {
+                const uint32_t st0 = q_count % kQStages;
+                ok &= mbar_wait(bar_kv, n_done & 1);
+                ok &= mbar_wait(bar_qdo + st0, (q_count / kQStages) & 1);
+                tc_fence_after();
+                issue_st(st0);
+                issue_dpt(st0);
+                for (int i = 0; i < n_q && ok; ++i) {
+                    const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
+                    ok &= mbar_wait(bar_p, ph);
+                    tc_fence_after();
+                    issue_dv(st, i > 0);
+                    if (i + 1 < n_q) {                   // S^T of the next query tile queues up behind dV
+                        ok &= mbar_wait(bar_qdo + st1, ((qc + 1) / kQStages) & 1);
+                        tc_fence_after();
+                        issue_st(st1);
+                    }
+                    ok &= mbar_wait(bar_ds, ph);
+                    tc_fence_after();
+                    issue_dq();
+                    issue_dk(st, i > 0);
+                    if (i + 1 < n_q) issue_dpt(st1);     // Q, dO of the next tile arrived before its S^T was issued
+                    else tc_commit(bar_acc);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            q_count += n_q;
+            ++n_done;
+            if (!ok) break;
+            continue;
+        }
+        // Query tile i of this item rides ring stage (q_count at item start + i) mod 3; the k-th use of a stage completes
+        // phase k of its barrier.  Tiles are fetched two ahead of the one being processed.
+        auto fetch_qdo = [&](int i, uint32_t stage) {    // warps 2 and 3 fetch Q and dO of query tile i; one thread announces the bytes
+            if (warp == 2) {
+                if ((tid & 31) == 0) mbar_expect_tx(bar_qdo + stage, 2 * kTileBytes);
+                load_tile(sQ + stage * kTileBytes, &map_q, bar_qdo + stage, src, i * kTile, n_sel, h, b, P.H);
+            } else if (warp == 3) {
+                load_tile(sdO + stage * kTileBytes, &map_do, bar_qdo + stage, src_do, i * kTile, n_sel, h, b, P.H);
+            }
+        };
         // plain loads first (row statistics, forward output, the variate this thread's key row scatters to): they are in
         // flight while the tile fetches are issued
         const int key = jt * kTile + row;               // this thread's key row
         const bool key_valid = key < n_sel;
+        const uint32_t st0 = q_count % kQStages;
         const float lse_first = load_lse(b, h, row);
+        const float lse_second = n_q > 1 ? load_lse(b, h, kTile + row) : 0.f;
         uint4 o_cur[4], o_next[4];
         float dl_cur = load_delta(b, h, row), dl_next = 0.f;
         if (!use_delta) load_o(b, h, row, o_cur);
         const int n_out = key_valid ? (sel ? sel[key] : key) : 0;
-        {   // every MMA of the previous item has completed: K, V and both Q/dO stages are free.  Warps 0 .. 3 fetch K, V, Q, dO side
-            // by side (each looks up its own gather rows); the byte counts are announced by thread 0, and a barrier phase
-            // cannot complete before that arrival, whichever comes first.
-            const uint32_t st0 = q_count & 1;
-            if (tid == 0) {
-                mbar_expect_tx(bar_kv, 2 * kTileBytes);
-                mbar_expect_tx(bar_qdo + st0, 2 * kTileBytes);
-            }
+        {   // every MMA of the previous item has completed: K, V and every Q/dO stage are free.  Warps 0 .. 3 fetch K, V, Q, dO
+            // side by side (each looks up its own gather rows); a barrier phase cannot complete before the thread that
+            // announces its bytes has arrived, whichever comes first.
+            if (tid == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
             if (warp == 0) load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
             else if (warp == 1) load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            else if (warp == 2) load_tile(sQ + st0 * kTileBytes, &map_q, bar_qdo + st0, src, 0, n_sel, h, b, P.H);
-            else if (warp == 3) load_tile(sdO + st0 * kTileBytes, &map_do, bar_qdo + st0, src_do, 0, n_sel, h, b, P.H);
+            fetch_qdo(0, st0);
+            if (n_q > 1) fetch_qdo(1, (st0 + 1) % kQStages);
         }
-        if (half == 0) s_stat[(q_count & 1) * kTile + row] = lse_first;
+        if (half == 0) {
+            s_stat[st0 * kTile + row] = lse_first;
+            if (n_q > 1) s_stat[((st0 + 1) % kQStages) * kTile + row] = lse_second;
+        }
         if (!zeros_written) write_zero_rows();
+        worker_sync();                                   // row statistics of the first tiles visible
 
+        // drains dQ of query tile `i` (complete on bar_g, phase `ph`) from tensor memory: lane = query row, this thread
+        // takes 32 of the 64 head-dimension columns
+        auto drain_dq = [&](int i, uint32_t ph) {
+            ok &= mbar_wait(bar_g, ph);
+            tc_fence_after();
+            const int qrow = i * kTile + row;
+            float dqv[32];
+            tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
+            tmem_ld_wait();
+            if (single_tile) {                           // final value: straight to the full-layout gradient, scaled, bf16
+                if (qrow < n_sel && half * 32 < P.D) {
+                    const int n = sel ? sel[qrow] : qrow;
+                    __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4*>(dst + q * 8) =
+                            make_uint4(pack2(dqv[8 * q + 0] * P.scale, dqv[8 * q + 1] * P.scale), pack2(dqv[8 * q + 2] * P.scale, dqv[8 * q + 3] * P.scale),
+                                       pack2(dqv[8 * q + 4] * P.scale, dqv[8 * q + 5] * P.scale), pack2(dqv[8 * q + 6] * P.scale, dqv[8 * q + 7] * P.scale));
+                }
+            } else {                                     // rows past n_sel are exact zeros (their probabilities are zero)
+                unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    *reinterpret_cast<float4*>(rowp + ((x ^ (row & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
+                fence_proxy_async_smem();
+            }
+            tc_fence_before();
+        };
+        auto reduce_dq = [&](int i) {                    // one bulk reduce-add per half: dq_acc[b, 128 i .., h, 32 half ..] += tile (one thread)
+            tma_reduce_add_4d(&map_acc, sDQ, 0, h, i * kTile, b);
+            tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, h, i * kTile, b);
+            bulk_commit_group();
+        };
+
+        // The query loop is a two-phase pipeline.  Phase A turns S^T into P^T while the tensor core still runs dK, dP^T of the
+        // previous tile; once P^T is in shared memory dV and the next S^T are issued.  Phase B turns dP^T into dS^T while
+        // those run; then dQ, dK and the next dP^T are issued.  dQ of a tile is drained one phase later, behind the next
+        // tile's phase A, when it is surely complete.
         for (int i = 0; i < n_q; ++i, ++q_count) {
-            const uint32_t st = q_count & 1, ph = q_count & 1;
-            float next_lse = 0.f;
+            const uint32_t st = q_count % kQStages, ph = q_count & 1;
+            const uint32_t st1 = (q_count + 1) % kQStages, st2 = (q_count + 2) % kQStages;
+            float lse_ahead = 0.f;
+            if (i + 2 < n_q) lse_ahead = load_lse(b, h, (i + 2) * kTile + row);       // lands while this tile is processed
             if (i + 1 < n_q) {
-                next_lse = load_lse(b, h, (i + 1) * kTile + row);        // both land while this tile is processed
                 dl_next = load_delta(b, h, (i + 1) * kTile + row);
                 if (!use_delta) load_o(b, h, (i + 1) * kTile + row, o_next);
-            }
-            if (tid == 0 && i == 0) {                    // later tiles: issued right behind the previous tile's products
-                ok &= mbar_wait(bar_kv, n_done & 1);
-                ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
-                tc_fence_after();
-                issue_scores(st);
             }
             if (use_delta) {
                 s_dpart[half * kTile + row] = dl_cur;    // half 1 holds the value, half 0 contributes zero
             } else {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
-                ok &= mbar_wait(bar_qdo + st, (q_count >> 1) & 1);
+                ok &= mbar_wait(bar_qdo + st, (q_count / kQStages) & 1);
                 const unsigned char* do_row = sdO + st * kTileBytes + row * kRowBytes;
                 float part = 0.f;
 #pragma unroll
@@ -339,110 +466,87 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     part += dot8(o_cur[x], *reinterpret_cast<const uint4*>(do_row + (((half * 4 + x) ^ (row & 7)) << 4)));
                 s_dpart[half * kTile + row] = part;
             }
-            __syncthreads();                             // row statistics of this stage visible
+
+            // ---- phase A: P^T of this thread's key row, its 64 queries (kept in registers for phase B) ----------
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
-            if (i + 1 < n_q) {                           // scores of this tile done => every product of the previous tile is done:
-                if (tid == 0) mbar_expect_tx(bar_qdo + (st ^ 1), 2 * kTileBytes);      // the other Q / dO stage is free
-                if (warp == 2) load_tile(sQ + (st ^ 1) * kTileBytes, &map_q, bar_qdo + (st ^ 1), src, (i + 1) * kTile, n_sel, h, b, P.H);
-                else if (warp == 3) load_tile(sdO + (st ^ 1) * kTileBytes, &map_do, bar_qdo + (st ^ 1), src_do, (i + 1) * kTile, n_sel, h, b, P.H);
-            }
-
-            // ---- P^T and dS^T: this thread's key row, its 64 queries -----------------------------------------
-            const float* lse2 = s_stat + st * kTile + half * 64;
-            const float* dlt = s_dpart + half * 64;
+            float pv[64];
+            {
+                const float* lse2 = s_stat + st * kTile + half * 64;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                float sv[32], dp[32];
-                tmem_ld32(tm_st + lane_sel + half * 64 + c * 32, sv);
-                tmem_ld32(tm_dpt + lane_sel + half * 64 + c * 32, dp);
-                tmem_ld_wait();
+                for (int c = 0; c < 2; ++c) {
+                    float sv[32];
+                    tmem_ld32(tm_st + lane_sel + half * 64 + c * 32, sv);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < 32; x += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 32 + x);
-                    const float4 da = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
-                    const float4 db = *reinterpret_cast<const float4*>(dlt + kTile + c * 32 + x);
-                    const float4 d4 = make_float4(da.x + db.x, da.y + db.y, da.z + db.z, da.w + db.w);
-                    const float p0 = fast_exp2(fmaf(sv[x + 0], P.scale_log2, -l4.x)), p1 = fast_exp2(fmaf(sv[x + 1], P.scale_log2, -l4.y));
-                    const float p2 = fast_exp2(fmaf(sv[x + 2], P.scale_log2, -l4.z)), p3 = fast_exp2(fmaf(sv[x + 3], P.scale_log2, -l4.w));
-                    sv[x + 0] = p0; sv[x + 1] = p1; sv[x + 2] = p2; sv[x + 3] = p3;
-                    dp[x + 0] = p0 * (dp[x + 0] - d4.x); dp[x + 1] = p1 * (dp[x + 1] - d4.y);
-                    dp[x + 2] = p2 * (dp[x + 2] - d4.z); dp[x + 3] = p3 * (dp[x + 3] - d4.w);
+                    for (int x = 0; x < 32; x += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 32 + x);
+                        pv[c * 32 + x + 0] = key_valid ? fast_exp2(fmaf(sv[x + 0], P.scale_log2, -l4.x)) : 0.f;    // rows past n_sel hold zero
+                        pv[c * 32 + x + 1] = key_valid ? fast_exp2(fmaf(sv[x + 1], P.scale_log2, -l4.y)) : 0.f;    // keys: they must not count
+                        pv[c * 32 + x + 2] = key_valid ? fast_exp2(fmaf(sv[x + 2], P.scale_log2, -l4.z)) : 0.f;
+                        pv[c * 32 + x + 3] = key_valid ? fast_exp2(fmaf(sv[x + 3], P.scale_log2, -l4.w)) : 0.f;
+                    }
+                    store_chunk32(sPt, row, half * 64 + c * 32, pv + c * 32);
                 }
-                if (!key_valid) {                        // rows past n_sel hold zero keys: their probabilities must not count
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) { sv[x] = 0.f; dp[x] = 0.f; }
-                }
-                store_chunk32(sPt, row, half * 64 + c * 32, sv);
-                store_chunk32(sdSt, row, half * 64 + c * 32, dp);
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            if (tid == 0) bulk_wait_group_read0();       // the previous tile's dQ reduction has read its shared-memory tile
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-                const uint64_t mq = umma_desc_advance(m_q0, st * kTileBytes), mdo = umma_desc_advance(m_do0, st * kTileBytes);
+            mbar_arrive(bar_p);                          // dV and the next S^T may go
+            if (i > 0) {                                 // dQ of the previous tile, into the shared-memory tile of the reduction
+                if (tid == 0) bulk_wait_group_read0();   // once the reduction before it has read that tile
+                worker_sync();
+                drain_dq(i - 1, ph ^ 1);
+            }
+
+            // ---- phase B: dS^T = P^T o (dP^T - Delta) ----------------------------------------------------------
+            ok &= mbar_wait(bar_dp, ph);                 // dP^T done => every product of the previous tile is done: its ring stage is free
+            tc_fence_after();
+            if (i + 2 < n_q) fetch_qdo(i + 2, st2);
+            {
+                const float* dlt = s_dpart + half * 64;
 #pragma unroll
-                for (int ks = 0; ks < kTile / 16; ++ks)              // reduction over the 128 keys: dQ_i = dS K, first: it is drained
-                    tc_mma_bf16(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
-                tc_commit(bar_g);                                    // while the other products and the next scores run
-                const uint32_t acc_on = i > 0;
+                for (int c = 0; c < 2; ++c) {
+                    float dp[32];
+                    tmem_ld32(tm_dpt + lane_sel + half * 64 + c * 32, dp);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int ks = 0; ks < kTile / 16; ++ks) {            // reduction over the 128 queries
-                    const uint32_t a_off = (ks >> 2) * kTileBytes + (ks & 3) * 32;
-                    tc_mma_bf16(tm_dv, umma_desc_advance(d_pt, a_off), umma_desc_advance(mdo, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
-                    tc_mma_bf16(tm_dk, umma_desc_advance(d_dst, a_off), umma_desc_advance(mq, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
-                }
-                if (i + 1 == n_q) tc_commit(bar_acc);
-                if (i + 1 < n_q) {                       // S^T, dP^T of the next query tile queue up behind these products
-                    ok &= mbar_wait(bar_qdo + (st ^ 1), ((q_count + 1) >> 1) & 1);
-                    tc_fence_after();
-                    issue_scores(st ^ 1);
+                    for (int x = 0; x < 32; x += 4) {
+                        const float4 da = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
+                        const float4 db = *reinterpret_cast<const float4*>(dlt + kTile + c * 32 + x);
+                        dp[x + 0] = pv[c * 32 + x + 0] * (dp[x + 0] - (da.x + db.x));
+                        dp[x + 1] = pv[c * 32 + x + 1] * (dp[x + 1] - (da.y + db.y));
+                        dp[x + 2] = pv[c * 32 + x + 2] * (dp[x + 2] - (da.z + db.z));
+                        dp[x + 3] = pv[c * 32 + x + 3] * (dp[x + 3] - (da.w + db.w));
+                    }
+                    store_chunk32(sdSt, row, half * 64 + c * 32, dp);
                 }
             }
+            if (i + 2 < n_q && half == 0) s_stat[st2 * kTile + row] = lse_ahead;       // read two tiles from now, behind several barriers
             if (i + 1 < n_q) {
-                if (half == 0) s_stat[(st ^ 1) * kTile + row] = next_lse;        // read only after the next top-of-loop barrier
                 dl_cur = dl_next;
                 if (!use_delta) {
 #pragma unroll
                     for (int x = 0; x < 4; ++x) o_cur[x] = o_next[x];
                 }
             }
-            ok &= mbar_wait(bar_g, ph);
-            tc_fence_after();
-            {   // dQ_i: tensor-memory lane = query row; this thread drains 32 of the 64 head-dimension columns
-                const int qrow = i * kTile + row;
-                const bool qv = qrow < n_sel;
-                float dqv[32];
-                tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
-                tmem_ld_wait();
-                if (single_tile) {                       // final value: straight to the full-layout gradient, scaled, bf16
-                    if (qv && half * 32 < P.D) {
-                        const int n = sel ? sel[qrow] : qrow;
-                        __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4*>(dst + q * 8) =
-                                make_uint4(pack2(dqv[8 * q + 0] * P.scale, dqv[8 * q + 1] * P.scale), pack2(dqv[8 * q + 2] * P.scale, dqv[8 * q + 3] * P.scale),
-                                           pack2(dqv[8 * q + 4] * P.scale, dqv[8 * q + 5] * P.scale), pack2(dqv[8 * q + 6] * P.scale, dqv[8 * q + 7] * P.scale));
-                    }
-                } else {                                 // rows past n_sel are exact zeros (their probabilities are zero)
-                    unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
-#pragma unroll
-                    for (int x = 0; x < 8; ++x)
-                        *reinterpret_cast<float4*>(rowp + ((x ^ (row & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
-                    fence_proxy_async_smem();
-                }
-            }
+            fence_proxy_async_smem();
             tc_fence_before();
-            ok = __syncthreads_and(ok);
+            mbar_arrive(bar_ds);                         // dQ, dK and the next dP^T may go
+            ok = worker_sync_and(ok);                    // a wait gave up somewhere among the workers: stop
             if (!ok) break;
-            if (!single_tile && tid == 0) {              // one bulk reduce-add per half: dq_acc[b, 128 i .., h, 32 half ..] += tile
-                tma_reduce_add_4d(&map_acc, sDQ, 0, h, i * kTile, b);
-                tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, h, i * kTile, b);
-                bulk_commit_group();
-            }
+            if (tid == 0 && i > 0) reduce_dq(i - 1);     // every thread's piece of the previous dQ tile is in shared memory
+        }
+        if (!ok) break;
+
+        // dQ of the last query tile
+        if (!single_tile) {
+            if (tid == 0) bulk_wait_group_read0();
+            worker_sync();
+        }
+        drain_dq(n_q - 1, (q_count - 1) & 1);
+        if (!single_tile) {
+            worker_sync();
+            if (tid == 0) reduce_dq(n_q - 1);
         }
 
         ok &= mbar_wait(bar_acc, n_done & 1);
@@ -470,20 +574,20 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                    pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
             }
             tc_fence_before();
-            __syncthreads();        // the accumulators are read out before the next item's products overwrite them
+            worker_sync();          // everyone is past this item's statistics and accumulators
         }
         if (P.convert_here && !single_tile && ok) {   // dQ' of this (instance, head) is complete once all its key tiles are: the last one converts it
-            int* flag = reinterpret_cast<int*>(smem_dyn + 60);
+            int* flag = reinterpret_cast<int*>(smem_dyn + 92);
             if (tid == 0) {
                 bulk_wait_group0();                      // this item's reductions have landed
                 __threadfence();
                 *flag = atomicAdd(P.tile_done + b * P.H + h, 1) == n_q - 1;
             }
-            __syncthreads();
+            worker_sync();
             if (*flag) {
                 __threadfence();
                 const int chunks_head = P.D / 8;         // 16-byte output chunks per row
-                for (int idx = tid; idx < n_sel * chunks_head; idx += blockDim.x) {
+                for (int idx = tid; idx < n_sel * chunks_head; idx += kBwdWorkers) {
                     const int j = idx / chunks_head, dc = idx - j * chunks_head;
                     const float4* acc = reinterpret_cast<const float4*>(P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * kDP) + dc * 2;
                     const float4 a0 = __ldcg(acc), a1 = __ldcg(acc + 1);
@@ -493,11 +597,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                    pack2(a1.x * P.scale, a1.y * P.scale), pack2(a1.z * P.scale, a1.w * P.scale));
                 }
             }
-            __syncthreads();        // `flag` is free for the next item
+            worker_sync();          // `flag` is free for the next item
         }
         ++n_done;
     }
-    if (!zeros_written) write_zero_rows();           // every item of this CTA was skipped (short instances)
+    if (!zeros_written && tid < kBwdWorkers) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
     tc_fence_before();
