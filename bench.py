@@ -183,8 +183,10 @@ def time_region(torch, fn, steps, dist_barrier):
     dist_barrier()
     torch.cuda.synchronize()
     start.record()
+    t0 = time.perf_counter()
     for i in range(steps):
         fn(i)
+    time_region.host_ms = (time.perf_counter() - t0) * 1e3          # host time spent issuing the K steps
     stop.record()
     torch.cuda.synchronize()
     dist_barrier()
@@ -295,6 +297,7 @@ def run_gpu(args):
         time.sleep(0.3)
     launches0 = vd.vardrop_launch_count()
     ms = time_region(torch, lambda i: path.step(i % slots), args.steps, barrier)
+    host_ms = time_region.host_ms
     launches = vd.vardrop_launch_count() - launches0
     # ---- same K steps with the per-kernel event timer armed (durations for the roofline) ----------------------
     vd.vardrop_profile_enable(True)
@@ -344,7 +347,7 @@ def run_gpu(args):
     line = {
         "metric": METRIC, "value": dist_util.aggregate_throughput(w.tokens, world, ms / args.steps * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "host_issue_ms_per_step": host_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 attention (fp32 accumulate), fp32 FFT, integer grouping", "data": "synthetic",
         "config": {"workload": f"{w.name}: B={w.B} N={w.N} L={w.L} k={w.k} rate={w.rate} H={w.H} D={w.D}",
                    "kept_tokens": n_sel, "groups": n_groups, "delta": 1.0 - n_sel / w.N,

@@ -79,11 +79,19 @@ def load() -> C.CDLL:
 
 
 def _ptr(t):
-    return None if t is None else C.c_void_p(t.data_ptr())
+    return None if t is None else t.data_ptr()        # a plain int converts to void* without a ctypes object per argument
+
+
+try:
+    _raw_stream = torch._C._cuda_getCurrentRawStream    # the stream handle without building a Stream object
+except AttributeError:                                   # pragma: no cover
+    _raw_stream = None
 
 
 def _stream():
-    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if _raw_stream is not None:
+        return _raw_stream(torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 def _check(status: int, where: str):

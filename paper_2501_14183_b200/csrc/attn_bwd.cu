@@ -100,7 +100,12 @@ struct BwdParams {
 };
 
 constexpr int kBwdWorkers = 256;       // two threads per tensor-memory lane: each takes one 64-column half
-constexpr int kBwdThreads = kBwdWorkers + 32;   // plus one warp whose first lane issues every tensor-core product
+constexpr int kBwdThreads = kBwdWorkers + 128; // plus a third warpgroup: its first warp's first lane issues every tensor-core product,
+                                               // the rest of it only gives its registers to the workers
+// Register split (setmaxnreg works on whole warpgroups): the kernel is launched with 384 x 168 = 64512 registers; the
+// third warpgroup keeps 104 a thread and the two worker warpgroups take 200: 256 x 200 + 128 x 104 = 64512.
+constexpr int kBwdWorkerRegs = 200;
+constexpr int kBwdIssuerRegs = 104;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr int kQStages = 3;            // ring of query-tile operands (Q and dO), fetched two tiles ahead
 constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 2 * kQStages * kTileBytes /*Q, dO ring*/ +
@@ -134,6 +139,18 @@ __device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0
     const int chunk0 = (c0 & 63) >> 3;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
+        const uint4 w = make_uint4(pack2(v[8 * q + 0], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                   pack2(v[8 * q + 6], v[8 * q + 7]));
+        *reinterpret_cast<uint4*>(panel + (((chunk0 + q) ^ (r & 7)) << 4)) = w;
+    }
+}
+
+// 16 consecutive columns (c0 a multiple of 16) of row r of the same tile layout
+__device__ __forceinline__ void store_chunk16(unsigned char* tile, int r, int c0, const float* v) {
+    unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
+    const int chunk0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
         const uint4 w = make_uint4(pack2(v[8 * q + 0], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
                                    pack2(v[8 * q + 6], v[8 * q + 7]));
         *reinterpret_cast<uint4*>(panel + (((chunk0 + q) ^ (r & 7)) << 4)) = w;
@@ -323,24 +340,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         return a0.x * g0.x + a0.y * g0.y + a1.x * g1.x + a1.y * g1.y + a2.x * g2.x + a2.y * g2.y + a3.x * g3.x + a3.y * g3.y;
     };
 
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const int jt = item % n_t_max;
-        const int h = (item / n_t_max) % P.H;
-        const int b = item / (n_t_max * P.H);
-        const int srow = P.S > 1 ? b : 0;
-        n_sel = P.S > 1 ? P.n_sel[srow] : kept_shared;
-        const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
-        if (jt >= n_q) continue;
-        const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
-        use_delta = P.delta != nullptr && n_q > 1;                 // precomputed Delta exists only when there are several key tiles
-        const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
-        TileSource src = P.src, src_do = P.src_do;
-        if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
-        if (warp == kBwdWorkers / 32) {
-            // The issuing warp: its first lane queues the products as their operands become ready.  The workers announce
-            // P^T and dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and
-            // the next dP^T while they compute the next P^T.
-            if ((tid & 31) == 0) {
+    if (warp >= kBwdWorkers / 32) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kBwdIssuerRegs));
+        // The issuing warp: its first lane queues the products as their operands become ready.  The workers announce P^T and
+        // dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and the next
+        // dP^T while they compute the next P^T.  The other warps of this warpgroup have nothing to do.
+        if (tid == kBwdWorkers) {
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const int jt = item % n_t_max;
+                const int b = item / (n_t_max * P.H);
+                const int kept = P.S > 1 ? P.n_sel[b] : kept_shared;
+                const int n_q = (kept + kTile - 1) / kTile;
+                if (jt >= n_q) continue;
                 const uint32_t st0 = q_count % kQStages;
                 ok &= mbar_wait(bar_kv, n_done & 1);
                 ok &= mbar_wait(bar_qdo + st0, (q_count / kQStages) & 1);
@@ -364,13 +375,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (i + 1 < n_q) issue_dpt(st1);     // Q, dO of the next tile arrived before its S^T was issued
                     else tc_commit(bar_acc);
                 }
+                q_count += n_q;
+                ++n_done;
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            q_count += n_q;
-            ++n_done;
-            if (!ok) break;
-            continue;
         }
+    } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kBwdWorkerRegs));
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int jt = item % n_t_max;
+        const int h = (item / n_t_max) % P.H;
+        const int b = item / (n_t_max * P.H);
+        const int srow = P.S > 1 ? b : 0;
+        n_sel = P.S > 1 ? P.n_sel[srow] : kept_shared;
+        const int n_q = (n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
+        if (jt >= n_q) continue;
+        const bool single_tile = n_q == 1;     // one key tile: dQ' needs no accumulation across CTAs
+        use_delta = P.delta != nullptr && n_q > 1;                 // precomputed Delta exists only when there are several key tiles
+        const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
+        TileSource src = P.src, src_do = P.src_do;
+        if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
         // Query tile i of this item rides ring stage (q_count at item start + i) mod 3; the k-th use of a stage completes
         // phase k of its barrier.  Tiles are fetched two ahead of the one being processed.
         auto fetch_qdo = [&](int i, uint32_t stage) {    // warps 2 and 3 fetch Q and dO of query tile i; one thread announces the bytes
@@ -456,7 +479,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 if (!use_delta) load_o(b, h, (i + 1) * kTile + row, o_next);
             }
             if (use_delta) {
-                s_dpart[half * kTile + row] = dl_cur;    // half 1 holds the value, half 0 contributes zero
+                if (half == 1) s_dpart[row] = dl_cur;    // the complete value: phase B reads one array
             } else {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
                 ok &= mbar_wait(bar_qdo + st, (q_count / kQStages) & 1);
                 const unsigned char* do_row = sdO + st * kTileBytes + row * kRowBytes;
@@ -471,22 +494,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             ok &= mbar_wait(bar_s, ph);
             tc_fence_after();
             float pv[64];
-            {
+            {   // 16 queries at a time; the next piece is read from tensor memory while the current one is processed
                 const float* lse2 = s_stat + st * kTile + half * 64;
+                float sv[2][16];
+                tmem_ld16(tm_st + lane_sel + half * 64, sv[0]);
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    float sv[32];
-                    tmem_ld32(tm_st + lane_sel + half * 64 + c * 32, sv);
+                for (int c = 0; c < 4; ++c) {
                     tmem_ld_wait();
+                    if (c < 3) tmem_ld16(tm_st + lane_sel + half * 64 + (c + 1) * 16, sv[(c + 1) & 1]);
 #pragma unroll
-                    for (int x = 0; x < 32; x += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 32 + x);
-                        pv[c * 32 + x + 0] = key_valid ? fast_exp2(fmaf(sv[x + 0], P.scale_log2, -l4.x)) : 0.f;    // rows past n_sel hold zero
-                        pv[c * 32 + x + 1] = key_valid ? fast_exp2(fmaf(sv[x + 1], P.scale_log2, -l4.y)) : 0.f;    // keys: they must not count
-                        pv[c * 32 + x + 2] = key_valid ? fast_exp2(fmaf(sv[x + 2], P.scale_log2, -l4.z)) : 0.f;
-                        pv[c * 32 + x + 3] = key_valid ? fast_exp2(fmaf(sv[x + 3], P.scale_log2, -l4.w)) : 0.f;
+                    for (int x = 0; x < 16; x += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 16 + x);
+                        pv[c * 16 + x + 0] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 0], P.scale_log2, -l4.x)) : 0.f;    // rows past n_sel hold zero
+                        pv[c * 16 + x + 1] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 1], P.scale_log2, -l4.y)) : 0.f;    // keys: they must not count
+                        pv[c * 16 + x + 2] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 2], P.scale_log2, -l4.z)) : 0.f;
+                        pv[c * 16 + x + 3] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 3], P.scale_log2, -l4.w)) : 0.f;
                     }
-                    store_chunk32(sPt, row, half * 64 + c * 32, pv + c * 32);
+                    store_chunk16(sPt, row, half * 64 + c * 16, pv + c * 16);
                 }
             }
             fence_proxy_async_smem();
@@ -504,21 +528,34 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (i + 2 < n_q) fetch_qdo(i + 2, st2);
             {
                 const float* dlt = s_dpart + half * 64;
+                float dp[2][16];
+                tmem_ld16(tm_dpt + lane_sel + half * 64, dp[0]);
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    float dp[32];
-                    tmem_ld32(tm_dpt + lane_sel + half * 64 + c * 32, dp);
+                for (int c = 0; c < 4; ++c) {
                     tmem_ld_wait();
+                    if (c < 3) tmem_ld16(tm_dpt + lane_sel + half * 64 + (c + 1) * 16, dp[(c + 1) & 1]);
+                    float* d = dp[c & 1];
+                    if (use_delta) {                     // one array holds the complete Delta
 #pragma unroll
-                    for (int x = 0; x < 32; x += 4) {
-                        const float4 da = *reinterpret_cast<const float4*>(dlt + c * 32 + x);
-                        const float4 db = *reinterpret_cast<const float4*>(dlt + kTile + c * 32 + x);
-                        dp[x + 0] = pv[c * 32 + x + 0] * (dp[x + 0] - (da.x + db.x));
-                        dp[x + 1] = pv[c * 32 + x + 1] * (dp[x + 1] - (da.y + db.y));
-                        dp[x + 2] = pv[c * 32 + x + 2] * (dp[x + 2] - (da.z + db.z));
-                        dp[x + 3] = pv[c * 32 + x + 3] * (dp[x + 3] - (da.w + db.w));
+                        for (int x = 0; x < 16; x += 4) {
+                            const float4 da = *reinterpret_cast<const float4*>(dlt + c * 16 + x);
+                            d[x + 0] = pv[c * 16 + x + 0] * (d[x + 0] - da.x);
+                            d[x + 1] = pv[c * 16 + x + 1] * (d[x + 1] - da.y);
+                            d[x + 2] = pv[c * 16 + x + 2] * (d[x + 2] - da.z);
+                            d[x + 3] = pv[c * 16 + x + 3] * (d[x + 3] - da.w);
+                        }
+                    } else {                             // two partial sums, one per 32 head dimensions
+#pragma unroll
+                        for (int x = 0; x < 16; x += 4) {
+                            const float4 da = *reinterpret_cast<const float4*>(dlt + c * 16 + x);
+                            const float4 db = *reinterpret_cast<const float4*>(dlt + kTile + c * 16 + x);
+                            d[x + 0] = pv[c * 16 + x + 0] * (d[x + 0] - (da.x + db.x));
+                            d[x + 1] = pv[c * 16 + x + 1] * (d[x + 1] - (da.y + db.y));
+                            d[x + 2] = pv[c * 16 + x + 2] * (d[x + 2] - (da.z + db.z));
+                            d[x + 3] = pv[c * 16 + x + 3] * (d[x + 3] - (da.w + db.w));
+                        }
                     }
-                    store_chunk32(sdSt, row, half * 64 + c * 32, dp);
+                    store_chunk16(sdSt, row, half * 64 + c * 16, d);
                 }
             }
             if (i + 2 < n_q && half == 0) s_stat[st2 * kTile + row] = lse_ahead;       // read two tiles from now, behind several barriers
@@ -601,6 +638,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
         ++n_done;
     }
+    }   // workers
     if (!zeros_written && tid < kBwdWorkers) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
