@@ -440,17 +440,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             float dqv[32];
             tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
             tmem_ld_wait();
-            if (single_tile) {                           // final value: straight to the full-layout gradient, scaled, bf16
-                if (qrow < n_sel && half * 32 < P.D) {
-                    const int n = sel ? sel[qrow] : qrow;
-                    __nv_bfloat16* dst = P.dq + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + half * 32;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4*>(dst + q * 8) =
-                            make_uint4(pack2(dqv[8 * q + 0] * P.scale, dqv[8 * q + 1] * P.scale), pack2(dqv[8 * q + 2] * P.scale, dqv[8 * q + 3] * P.scale),
-                                       pack2(dqv[8 * q + 4] * P.scale, dqv[8 * q + 5] * P.scale), pack2(dqv[8 * q + 6] * P.scale, dqv[8 * q + 7] * P.scale));
-                }
-            } else {                                     // rows past n_sel are exact zeros (their probabilities are zero)
+            {                                            // rows past n_sel are exact zeros (their probabilities are zero)
                 unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
 #pragma unroll
                 for (int x = 0; x < 8; ++x)
@@ -575,43 +565,54 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
         if (!ok) break;
 
-        // dQ of the last query tile
+        // dQ of the last query tile: with several key tiles it joins the accumulator like the others
         if (!single_tile) {
             if (tid == 0) bulk_wait_group_read0();
             worker_sync();
-        }
-        drain_dq(n_q - 1, (q_count - 1) & 1);
-        if (!single_tile) {
+            drain_dq(n_q - 1, (q_count - 1) & 1);
             worker_sync();
             if (tid == 0) reduce_dq(n_q - 1);
         }
 
         ok &= mbar_wait(bar_acc, n_done & 1);
         tc_fence_after();
-        {   // dV, dK of this key tile: every thread takes part in the warp-collective loads, only valid key rows store
-            const bool store = ok && key_valid && half * 32 < P.D;
-            const size_t out = ((static_cast<size_t>(b) * P.N + n_out) * P.H + h) * P.D + half * 32;
-            float acc[32];
-            tmem_ld32(tm_dv + lane_sel + half * 32, acc);
-            tmem_ld_wait();
-            if (store) {
+        {   // dV, dK of this key tile (and dQ when this is the only key tile: key row = query row): every thread rounds its 32
+            // columns to bf16 into a staging tile (the P^T / dS^T tiles are free now), then eight threads write each 128-byte
+            // row of the full-layout gradients in one piece.
+            unsigned char* stage_dv = sPt;
+            unsigned char* stage_dk = sPt + kTileBytes;
+            unsigned char* stage_dq = sdSt;
+            int* s_nout = reinterpret_cast<int*>(sdSt + kTileBytes);           // variate of each key row, -1: no such row
+            auto stage = [&](unsigned char* tile, uint32_t tm, float mul) {
+                float acc[32];
+                tmem_ld32(tm + lane_sel + half * 32, acc);
+                tmem_ld_wait();
+                unsigned char* rowp = tile + row * kRowBytes;
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4*>(P.dv + out + q * 8) =
-                        make_uint4(pack2(acc[8 * q + 0], acc[8 * q + 1]), pack2(acc[8 * q + 2], acc[8 * q + 3]),
-                                   pack2(acc[8 * q + 4], acc[8 * q + 5]), pack2(acc[8 * q + 6], acc[8 * q + 7]));
-            }
-            tmem_ld32(tm_dk + lane_sel + half * 32, acc);
-            tmem_ld_wait();
-            if (store) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4*>(P.dk + out + q * 8) =
-                        make_uint4(pack2(acc[8 * q + 0] * P.scale, acc[8 * q + 1] * P.scale), pack2(acc[8 * q + 2] * P.scale, acc[8 * q + 3] * P.scale),
-                                   pack2(acc[8 * q + 4] * P.scale, acc[8 * q + 5] * P.scale), pack2(acc[8 * q + 6] * P.scale, acc[8 * q + 7] * P.scale));
-            }
+                    *reinterpret_cast<uint4*>(rowp + (((half * 4 + q) ^ (row & 7)) << 4)) =
+                        make_uint4(pack2(acc[8 * q + 0] * mul, acc[8 * q + 1] * mul), pack2(acc[8 * q + 2] * mul, acc[8 * q + 3] * mul),
+                                   pack2(acc[8 * q + 4] * mul, acc[8 * q + 5] * mul), pack2(acc[8 * q + 6] * mul, acc[8 * q + 7] * mul));
+            };
+            stage(stage_dv, tm_dv, 1.f);
+            stage(stage_dk, tm_dk, P.scale);
+            if (single_tile) stage(stage_dq, tm_dq, P.scale);                   // complete: bar_acc covers every product of the item
+            if (half == 0) s_nout[row] = key_valid ? n_out : -1;
             tc_fence_before();
-            worker_sync();          // everyone is past this item's statistics and accumulators
+            worker_sync();
+            const int c = tid & 7;
+            if (ok && c * 8 < P.D) {
+                for (int r = tid >> 3; r < kTile; r += kBwdWorkers / 8) {
+                    const int n = s_nout[r];
+                    if (n < 0) continue;
+                    const size_t out = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + c * 8;
+                    const int off = r * kRowBytes + ((c ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(P.dv + out) = *reinterpret_cast<const uint4*>(stage_dv + off);
+                    *reinterpret_cast<uint4*>(P.dk + out) = *reinterpret_cast<const uint4*>(stage_dk + off);
+                    if (single_tile) *reinterpret_cast<uint4*>(P.dq + out) = *reinterpret_cast<const uint4*>(stage_dq + off);
+                }
+            }
+            worker_sync();          // staging tiles, statistics and accumulators are free for the next item
         }
         if (P.convert_here && !single_tile && ok) {   // dQ' of this (instance, head) is complete once all its key tiles are: the last one converts it
             int* flag = reinterpret_cast<int*>(smem_dyn + 92);
