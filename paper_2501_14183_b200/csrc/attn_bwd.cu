@@ -126,26 +126,29 @@ __device__ __forceinline__ bool worker_sync_and(bool ok) {
     return r != 0;
 }
 
+// the same for the third warpgroup (128 threads, barrier 2)
+__device__ __forceinline__ void group3_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+__device__ __forceinline__ bool group3_sync_and(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "bar.red.and.pred p, 2, 128, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(ok))
+        : "memory");
+    return r != 0;
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
-// 32 consecutive columns (c0 a multiple of 32) of row r of a 128 x 128 bf16 tile stored as two 64-column panels
+// 16 consecutive columns (c0 a multiple of 16) of row r of a 128 x 128 bf16 tile stored as two 64-column panels
 // (128-byte swizzled rows)
-__device__ __forceinline__ void store_chunk32(unsigned char* tile, int r, int c0, const float* v) {
-    unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
-    const int chunk0 = (c0 & 63) >> 3;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const uint4 w = make_uint4(pack2(v[8 * q + 0], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
-                                   pack2(v[8 * q + 6], v[8 * q + 7]));
-        *reinterpret_cast<uint4*>(panel + (((chunk0 + q) ^ (r & 7)) << 4)) = w;
-    }
-}
-
-// 16 consecutive columns (c0 a multiple of 16) of row r of the same tile layout
 __device__ __forceinline__ void store_chunk16(unsigned char* tile, int r, int c0, const float* v) {
     unsigned char* panel = tile + (c0 >> 6) * kTileBytes + r * kRowBytes;
     const int chunk0 = (c0 & 63) >> 3;
@@ -167,7 +170,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     chain_release();
     // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
-    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 88)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 100)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
     // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
     // operand loads of its first work item, so the stores drain while those loads are in flight.
@@ -214,7 +217,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint64_t* bar_acc = bars + 7;                   // every product of the item complete: dV, dK final, operands free
     uint64_t* bar_p = bars + 8;                     // P^T of a query tile written by every worker thread
     uint64_t* bar_ds = bars + 9;                    // dS^T of a query tile written by every worker thread
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 80);
+    uint64_t* bar_conv = bars + 10;                 // the "last key tile of its (instance, head)" flag of an item is written
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 96);
     float* s_stat = reinterpret_cast<float*>(smem_dyn + 128);     // [3 stages][128] lse of the query tile, log2 domain
     float* s_dpart = s_stat + kQStages * kTile;                   // [2 halves][128] partial Delta = sum over 32 head dims of dO O
     unsigned char* sK = align_tiles(smem_dyn + 128 + (kQStages + 2) * kTile * sizeof(float));
@@ -245,6 +249,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         mbar_init(bar_acc, 1);
         mbar_init(bar_p, kBwdWorkers);
         mbar_init(bar_ds, kBwdWorkers);
+        mbar_init(bar_conv, 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_k);
@@ -272,6 +277,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     bool ok = true;
     uint32_t q_count = 0;       // query tiles consumed so far by this CTA: ring stage = q_count mod 3
     uint32_t n_done = 0;        // work items finished by this CTA (phase of bar_kv)
+    uint32_t n_conv = 0;        // items whose "last key tile" flag has been read (phase of bar_conv)
 
     // operand descriptors, built once and stepped by additions: K-major views for the scores and the P^T / dS^T panels,
     // MN-major views where the reduction runs over the rows of the tile
@@ -342,24 +348,31 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 
     if (warp >= kBwdWorkers / 32) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kBwdIssuerRegs));
-        // The issuing warp: its first lane queues the products as their operands become ready.  The workers announce P^T and
-        // dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and the next
-        // dP^T while they compute the next P^T.  The other warps of this warpgroup have nothing to do.
-        if (tid == kBwdWorkers) {
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int jt = item % n_t_max;
-                const int b = item / (n_t_max * P.H);
-                const int kept = P.S > 1 ? P.n_sel[b] : kept_shared;
-                const int n_q = (kept + kTile - 1) / kTile;
-                if (jt >= n_q) continue;
+        // The third warpgroup.  Its first thread queues the products as their operands become ready: the workers announce P^T
+        // and dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and the next
+        // dP^T while they compute the next P^T.  All four warps (one per quarter of the tensor-memory lanes) then take dQ of the
+        // tile out of tensor memory into the fp32 shared-memory tile, which one bulk reduction adds to the accumulator.
+        const bool issuer = tid == kBwdWorkers;
+        const int qrow_l = tid - kBwdWorkers;           // query row this thread drains
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int jt = item % n_t_max;
+            const int h = (item / n_t_max) % P.H;
+            const int b = item / (n_t_max * P.H);
+            const int kept = P.S > 1 ? P.n_sel[b] : kept_shared;
+            const int n_q = (kept + kTile - 1) / kTile;
+            if (jt >= n_q) continue;
+            const bool single_tile = n_q == 1;
+            if (issuer) {
                 const uint32_t st0 = q_count % kQStages;
                 ok &= mbar_wait(bar_kv, n_done & 1);
                 ok &= mbar_wait(bar_qdo + st0, (q_count / kQStages) & 1);
                 tc_fence_after();
                 issue_st(st0);
                 issue_dpt(st0);
-                for (int i = 0; i < n_q && ok; ++i) {
-                    const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
+            }
+            for (int i = 0; i < n_q; ++i) {
+                const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
+                if (issuer) {
                     ok &= mbar_wait(bar_p, ph);
                     tc_fence_after();
                     issue_dv(st, i > 0);
@@ -375,10 +388,48 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (i + 1 < n_q) issue_dpt(st1);     // Q, dO of the next tile arrived before its S^T was issued
                     else tc_commit(bar_acc);
                 }
-                q_count += n_q;
-                ++n_done;
+                __syncwarp();                            // the issuer's warp waits for it here instead of polling beside it
+                if (!single_tile) {                      // (a single key tile: the workers write dQ with dV and dK at the end)
+                    ok &= mbar_wait(bar_g, ph);
+                    tc_fence_after();
+                    if (issuer) bulk_wait_group_read0(); // the previous reduction has read the shared-memory tile
+                    group3_sync();
+                    float dqv[32];
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {     // rows past n_sel are exact zeros (their probabilities are zero)
+                        tmem_ld32(tm_dq + lane_sel + hf * 32, dqv);
+                        tmem_ld_wait();
+                        unsigned char* rowp = sDQ + hf * kTileBytes + qrow_l * kRowBytes;
+#pragma unroll
+                        for (int x = 0; x < 8; ++x)
+                            *reinterpret_cast<float4*>(rowp + ((x ^ (qrow_l & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
+                    }
+                    fence_proxy_async_smem();
+                    tc_fence_before();
+                    ok = group3_sync_and(ok);            // dQ is out of tensor memory: the next one may be issued
+                    if (issuer) {                        // one bulk reduce-add per half: dq_acc[b, 128 i .., h, 32 half ..] += tile
+                        tma_reduce_add_4d(&map_acc, sDQ, 0, h, i * kTile, b);
+                        tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, h, i * kTile, b);
+                        bulk_commit_group();
+                    }
+                    if (!ok) break;
+                }
             }
+            ok = group3_sync_and(ok);                    // the warpgroup leaves together if a wait gave up
+            if (!ok) break;
+            if (P.convert_here && !single_tile) {        // tell the workers whether this was the last key tile of its (instance, head)
+                if (issuer) {
+                    int* flag = reinterpret_cast<int*>(smem_dyn + 104);
+                    bulk_wait_group0();                  // this item's reductions have landed
+                    __threadfence();
+                    *flag = atomicAdd(P.tile_done + b * P.H + h, 1) == n_q - 1;
+                    mbar_arrive(bar_conv);
+                }
+            }
+            q_count += n_q;
+            ++n_done;
         }
+        if (tid == kBwdWorkers) bulk_wait_group0();      // the last dQ reductions have landed
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kBwdWorkerRegs));
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
@@ -431,37 +482,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         if (!zeros_written) write_zero_rows();
         worker_sync();                                   // row statistics of the first tiles visible
 
-        // drains dQ of query tile `i` (complete on bar_g, phase `ph`) from tensor memory: lane = query row, this thread
-        // takes 32 of the 64 head-dimension columns
-        auto drain_dq = [&](int i, uint32_t ph) {
-            ok &= mbar_wait(bar_g, ph);
-            tc_fence_after();
-            const int qrow = i * kTile + row;
-            float dqv[32];
-            tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
-            tmem_ld_wait();
-            {                                            // rows past n_sel are exact zeros (their probabilities are zero)
-                unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
-#pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    *reinterpret_cast<float4*>(rowp + ((x ^ (row & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
-                fence_proxy_async_smem();
-            }
-            tc_fence_before();
-        };
-        auto reduce_dq = [&](int i) {                    // one bulk reduce-add per half: dq_acc[b, 128 i .., h, 32 half ..] += tile (one thread)
-            tma_reduce_add_4d(&map_acc, sDQ, 0, h, i * kTile, b);
-            tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, h, i * kTile, b);
-            bulk_commit_group();
-        };
-
         // The query loop is a two-phase pipeline.  Phase A turns S^T into P^T while the tensor core still runs dK, dP^T of the
         // previous tile; once P^T is in shared memory dV and the next S^T are issued.  Phase B turns dP^T into dS^T while
         // those run; then dQ, dK and the next dP^T are issued.  dQ of a tile is drained one phase later, behind the next
         // tile's phase A, when it is surely complete.
         for (int i = 0; i < n_q; ++i, ++q_count) {
             const uint32_t st = q_count % kQStages, ph = q_count & 1;
-            const uint32_t st1 = (q_count + 1) % kQStages, st2 = (q_count + 2) % kQStages;
+            const uint32_t st2 = (q_count + 2) % kQStages;
             float lse_ahead = 0.f;
             if (i + 2 < n_q) lse_ahead = load_lse(b, h, (i + 2) * kTile + row);       // lands while this tile is processed
             if (i + 1 < n_q) {
@@ -506,11 +533,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar_p);                          // dV and the next S^T may go
-            if (i > 0) {                                 // dQ of the previous tile, into the shared-memory tile of the reduction
-                if (tid == 0) bulk_wait_group_read0();   // once the reduction before it has read that tile
-                worker_sync();
-                drain_dq(i - 1, ph ^ 1);
-            }
 
             // ---- phase B: dS^T = P^T o (dP^T - Delta) ----------------------------------------------------------
             ok &= mbar_wait(bar_dp, ph);                 // dP^T done => every product of the previous tile is done: its ring stage is free
@@ -561,18 +583,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             mbar_arrive(bar_ds);                         // dQ, dK and the next dP^T may go
             ok = worker_sync_and(ok);                    // a wait gave up somewhere among the workers: stop
             if (!ok) break;
-            if (tid == 0 && i > 0) reduce_dq(i - 1);     // every thread's piece of the previous dQ tile is in shared memory
         }
         if (!ok) break;
-
-        // dQ of the last query tile: with several key tiles it joins the accumulator like the others
-        if (!single_tile) {
-            if (tid == 0) bulk_wait_group_read0();
-            worker_sync();
-            drain_dq(n_q - 1, (q_count - 1) & 1);
-            worker_sync();
-            if (tid == 0) reduce_dq(n_q - 1);
-        }
 
         ok &= mbar_wait(bar_acc, n_done & 1);
         tc_fence_after();
@@ -599,7 +611,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (single_tile) stage(stage_dq, tm_dq, P.scale);                   // complete: bar_acc covers every product of the item
             if (half == 0) s_nout[row] = key_valid ? n_out : -1;
             tc_fence_before();
-            worker_sync();
+            ok = worker_sync_and(ok);                    // the workers go on (or give up) together
             const int c = tid & 7;
             if (ok && c * 8 < P.D) {
                 for (int r = tid >> 3; r < kTile; r += kBwdWorkers / 8) {
@@ -615,13 +627,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             worker_sync();          // staging tiles, statistics and accumulators are free for the next item
         }
         if (P.convert_here && !single_tile && ok) {   // dQ' of this (instance, head) is complete once all its key tiles are: the last one converts it
-            int* flag = reinterpret_cast<int*>(smem_dyn + 92);
-            if (tid == 0) {
-                bulk_wait_group0();                      // this item's reductions have landed
-                __threadfence();
-                *flag = atomicAdd(P.tile_done + b * P.H + h, 1) == n_q - 1;
-            }
-            worker_sync();
+            int* flag = reinterpret_cast<int*>(smem_dyn + 104);
+            ok &= mbar_wait(bar_conv, n_conv & 1);       // the third warpgroup has seen this item's reductions land and counted the tile
+            ++n_conv;
             if (*flag) {
                 __threadfence();
                 const int chunks_head = P.D / 8;         // 16-byte output chunks per row
@@ -642,7 +650,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     }   // workers
     if (!zeros_written && tid < kBwdWorkers) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
-    if (tid == 0) bulk_wait_group0();                // the last dQ reductions have landed
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
