@@ -419,10 +419,10 @@ int hash_rows_launch(const float* x, const vardrop_hash_cfg& c, int f_lo, int f_
     int per = (c.B + team - 1) / team;
     P.per_member = per + (per & 1);
     switch (c.L) {
-        case 96: return launch_rows<96, 8, 12, 8, 4>(P, stream);
+        case 96: return launch_rows<96, 8, 12, 8, 5>(P, stream);
         case 192: return launch_rows<192, 12, 16, 4, 3>(P, stream);
-        case 336: return launch_rows<336, 16, 21, 4, 3>(P, stream);
-        default: return launch_rows<720, 24, 30, 1, 3>(P, stream);
+        case 336: return launch_rows<336, 16, 21, 2, 4>(P, stream);
+        default: return launch_rows<720, 24, 30, 1, 4>(P, stream);
     }
 }
 
