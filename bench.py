@@ -222,6 +222,7 @@ def kernel_work(w, n_sel, selected=True):
         "hash_kernel": (w.B * w.N * w.L * 4 + w.N * (8 + 4 * w.k), None),
         "select_small_kernel": (w.N * (8 + 6 * 4), None),
         "select_count_kernel": (w.N * (8 + 4 * 4), None),
+        "select_group_kernel": (w.N * 6 * 4, None),
         "select_sample_kernel": (w.N * 4 * 4, None),
         "gather_kernel": (2 * 3 * kept * row, None),
         "attn_fwd_kernel": (3 * kept * row + kept * row + kept * w.H * 4, 4.0 * w.B * w.H * n_sel * n_sel * w.D),

@@ -11,7 +11,7 @@ namespace vardrop {
 
 // Kernel identities for the launch counter and the optional per-kernel event timer (vardrop_profile_*).
 enum KernelId {
-    K_HASH = 0, K_SELECT_SMALL, K_SELECT_COUNT, K_SELECT_SAMPLE, K_GATHER, K_ATTN_FWD, K_BWD_PREP, K_ATTN_BWD, K_BWD_CONVERT, K_COUNT
+    K_HASH = 0, K_SELECT_SMALL, K_SELECT_COUNT, K_SELECT_GROUP, K_SELECT_SAMPLE, K_GATHER, K_ATTN_FWD, K_BWD_PREP, K_ATTN_BWD, K_BWD_CONVERT, K_COUNT
 };
 // Wrap a kernel launch: counts it and, when the timer is armed, brackets it with a pair of CUDA events on `stream`.
 struct LaunchScope {

@@ -98,10 +98,58 @@ __device__ __forceinline__ bool last_cta_of_row(unsigned int* counter, unsigned 
     return last;
 }
 
+// Ordered compaction by one CTA: for every position p < N, in ascending order, `emit(p, set, before, payload)` is called
+// with (set, payload) = flag(p) and before = number of set flags at positions below p; returns the number of set flags.
+// Positions are dealt to the threads round-robin (position = batch base + chunk * kSelThreads + thread) and a batch of 32
+// chunks is handled with fully unrolled loops, so the (dependent) loads behind the 32 flags of a thread are coalesced and
+// all in flight at once instead of one memory round trip per position; a batch is ordered with warp ballots and one scan of
+// the per-warp counts.
+template <class FlagFn, class EmitFn>
+__device__ __forceinline__ int ordered_compact(int N, FlagFn flag, EmitFn emit) {
+    constexpr int kWarps = kSelThreads / 32;
+    __shared__ uint32_t s_mask[32 * kWarps];      // ballot of chunk k, warp w at [k * kWarps + w]: position order
+    __shared__ int s_excl[32 * kWarps];           // set flags of the batch before that (chunk, warp)
+    __shared__ int s_warp[kWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int done = 0;                                  // set flags of the batches before this one
+    for (int base = 0; base < N; base += 32 * kSelThreads) {
+        uint32_t bits = 0;                         // bit k: flag of position base + k * kSelThreads + thread
+        int payload[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const int p = base + k * kSelThreads + static_cast<int>(threadIdx.x);
+            payload[k] = 0;
+            if (p < N && flag(p, &payload[k])) bits |= 1u << k;
+        }
+        uint32_t mine = 0;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const uint32_t m = __ballot_sync(0xffffffffu, (bits >> k) & 1u);
+            if (lane == k) mine = m;
+        }
+        __syncthreads();                           // the tables of the previous batch are no longer read
+        s_mask[lane * kWarps + warp] = mine;
+        __syncthreads();
+        int total = 0;
+        const int cnt = __popc(s_mask[threadIdx.x]);               // kSelThreads = 32 * kWarps entries, one per thread
+        const int incl = block_scan_inclusive(cnt, s_warp, &total);
+        s_excl[threadIdx.x] = incl - cnt;
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const int p = base + k * kSelThreads + static_cast<int>(threadIdx.x);
+            if (p < N) {
+                const uint32_t m = s_mask[k * kWarps + warp];
+                emit(p, ((bits >> k) & 1u) != 0, done + s_excl[k * kWarps + warp] + __popc(m & ((1u << lane) - 1u)), payload[k]);
+            }
+        }
+        done += total;
+    }
+    return done;
+}
+
 __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectParams P) {
     __shared__ uint64_t skeys[kKeyChunk];
-    __shared__ int warp_sums[kSelThreads / 32];
-    __shared__ int flag;
     chain_wait();
     chain_release();
     const int s = blockIdx.z, N = P.N;
@@ -124,39 +172,66 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectP
         if (c_lt) atomicAdd(lt + n, c_lt);
         if (c_eq) atomicAdd(eq + n, c_eq);
     }
-    if (!last_cta_of_row(P.done1 + s, gridDim.x * gridDim.y, &flag)) return;
+}
 
-    // ---- the last CTA of this hash row: members, group heads -> ids and offsets, priorities ---------------
+// One CTA per hash row, after the counts are complete: members, group heads -> ids and offsets, priorities.
+__global__ void __launch_bounds__(kSelThreads) select_group_kernel(const SelectParams P) {
+    chain_wait();
+    chain_release();
+    const int s = blockIdx.x, N = P.N;
+    const int32_t* lt = P.lt + static_cast<size_t>(s) * N;
+    const int32_t* eq = P.eq + static_cast<size_t>(s) * N;
     int32_t* members = P.members + static_cast<size_t>(s) * N;
     int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
     int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
     uint32_t* prio = P.prio + static_cast<size_t>(s) * N;
-    for (int i = threadIdx.x; i < N; i += blockDim.x) members[__ldcg(lt + i) + __ldcg(eq + i)] = i;
-    __syncthreads();
-    // scan of head flags over sorted positions; thread t owns positions [t*per, (t+1)*per)
-    const int per = (N + kSelThreads - 1) / kSelThreads;
-    const int p_begin = min(N, static_cast<int>(threadIdx.x) * per), p_end = min(N, p_begin + per);
-    int heads = 0;
-    for (int p = p_begin; p < p_end; ++p) heads += (__ldcg(eq + members[p]) == 0);
-    int total_groups = 0;
-    int g = block_scan_inclusive(heads, warp_sums, &total_groups) - heads;   // groups before p_begin
-    for (int p = p_begin; p < p_end; ++p) {
-        const int nn = members[p];
-        if (__ldcg(eq + nn) == 0) { off[g] = p; ++g; }
-        gid[nn] = g - 1;
+    // every loop of this tail takes eight positions per thread at a time: the loads of a batch are issued together, so a
+    // batch costs one or two memory round trips instead of one per position
+    for (int base = 0; base < N; base += 8 * kSelThreads) {
+        int dst[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * kSelThreads + static_cast<int>(threadIdx.x);
+            dst[u] = i < N ? __ldcg(lt + i) + __ldcg(eq + i) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (dst[u] >= 0) members[dst[u]] = base + u * kSelThreads + static_cast<int>(threadIdx.x);
     }
+    __syncthreads();
+    // group heads over the sorted positions: the first member of every group has no equal key before it
+    const int total_groups = ordered_compact(
+        N, [&](int p, int* nn) { *nn = __ldcg(members + p); return __ldcg(eq + *nn) == 0; },
+        [&](int p, bool head, int before, int nn) {
+            if (head) off[before] = p;
+            gid[nn] = before - (head ? 0 : 1);           // heads at or below p, minus one
+        });
     for (int i = total_groups + threadIdx.x; i <= N; i += blockDim.x) off[i] = N;
     if (threadIdx.x == 0) P.n_groups[s] = total_groups;
     __syncthreads();
-    for (int p = threadIdx.x; p < N; p += blockDim.x) {
-        const int nn = members[p];
-        prio[p] = philox4x32_10_word0(static_cast<uint32_t>(__ldcg(eq + nn)), static_cast<uint32_t>(gid[nn]), static_cast<uint32_t>(s),
-                                      P.step, P.seed_lo, P.seed_hi);
+    for (int base = 0; base < N; base += 8 * kSelThreads) {
+        int nn[8], rank[8], g[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int p = base + u * kSelThreads + static_cast<int>(threadIdx.x);
+            nn[u] = p < N ? __ldcg(members + p) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            rank[u] = __ldcg(eq + nn[u]);
+            g[u] = __ldcg(gid + nn[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int p = base + u * kSelThreads + static_cast<int>(threadIdx.x);
+            if (p < N)
+                prio[p] = philox4x32_10_word0(static_cast<uint32_t>(rank[u]), static_cast<uint32_t>(g[u]), static_cast<uint32_t>(s), P.step,
+                                              P.seed_lo, P.seed_hi);
+        }
     }
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const SelectParams P) {
-    __shared__ int warp_sums[kSelThreads / 32];
     __shared__ int flag;
     chain_wait();
     chain_release();
@@ -184,15 +259,12 @@ __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const Select
     // ---- the last CTA of this hash row: compaction of the kept variates in ascending index order --------
     int32_t* sel = P.sel_idx + static_cast<size_t>(s) * N;
     int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
-    const int per = (N + kSelThreads - 1) / kSelThreads;
-    const int n_begin = min(N, static_cast<int>(threadIdx.x) * per), n_end = min(N, n_begin + per);
-    int cnt = 0;
-    for (int i = n_begin; i < n_end; ++i) cnt += __ldcg(keep + i);
-    int total = 0;
-    int pos = block_scan_inclusive(cnt, warp_sums, &total) - cnt;
-    for (int i = n_begin; i < n_end; ++i) {
-        if (__ldcg(keep + i)) { sel[pos] = i; inv[i] = pos; ++pos; } else inv[i] = -1;
-    }
+    const int total = ordered_compact(
+        N, [&](int i, int*) { return __ldcg(keep + i) != 0; },
+        [&](int i, bool kept, int before, int) {
+            if (kept) sel[before] = i;
+            inv[i] = kept ? before : -1;
+        });
     for (int i = total + threadIdx.x; i < N; i += blockDim.x) sel[i] = -1;
     if (threadIdx.x == 0) P.n_sel[s] = total;
 }
@@ -425,6 +497,8 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
     cudaError_t err;
     { LaunchScope ls_(K_SELECT_COUNT, stream); err = launch_chained(select_count_kernel, grid1, dim3(kSelThreads), 0, stream, P); }
     if (int st = check_cuda(err, "select: count launch")) return st;
+    { LaunchScope ls_(K_SELECT_GROUP, stream); err = launch_chained(select_group_kernel, dim3(c.S), dim3(kSelThreads), 0, stream, P); }
+    if (int st = check_cuda(err, "select: group launch")) return st;
     const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
     { LaunchScope ls_(K_SELECT_SAMPLE, stream); err = launch_chained(select_sample_kernel, grid2, dim3(kSelThreads), 0, stream, P); }
     return check_cuda(err, "select: sample launch");

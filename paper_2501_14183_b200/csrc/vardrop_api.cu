@@ -46,7 +46,7 @@ bool g_prof_on = false;
 long long g_launches = 0;
 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_events[K_COUNT];   // pairs recorded since the timer was armed
 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_free;              // pairs ready for reuse
-const char* const g_kernel_names[K_COUNT] = {"hash_kernel", "select_small_kernel", "select_count_kernel", "select_sample_kernel", "gather_kernel",
+const char* const g_kernel_names[K_COUNT] = {"hash_kernel", "select_small_kernel", "select_count_kernel", "select_group_kernel", "select_sample_kernel", "gather_kernel",
                                              "attn_fwd_kernel", "bwd_prep_kernel", "attn_bwd_kernel", "bwd_convert_kernel"};
 }  // namespace
 

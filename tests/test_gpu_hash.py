@@ -45,6 +45,7 @@ SHAPES = [
     (4, 21, 96, 2, 0), (1, 1, 96, 3, 0), (3, 37, 96, 3, 0), (32, 50, 96, 3, 0), (5, 33, 336, 4, 0), (16, 9, 720, 5, 0),
     (7, 19, 720, 5, 0), (2, 13, 48, 2, 0), (3, 11, 30, 2, 0), (2, 5, 14, 1, 0), (4, 8, 64, 3, 0), (3, 6, 2048, 5, 0),
     (70, 3, 96, 3, 0), (4, 21, 96, 2, 1), (3, 10, 336, 4, 1), (5, 7, 720, 5, 1), (1, 300, 96, 3, 0), (2, 4, 210, 3, 0),
+    (6, 17, 192, 3, 0), (9, 40, 192, 4, 0), (17, 23, 336, 4, 0), (2, 1300, 96, 3, 0), (33, 300, 96, 3, 0),
 ]
 
 
@@ -130,3 +131,20 @@ def test_hash_argument_errors():
     with pytest.raises(vd.VardropError) as e:
         vd.vardrop_hash(None, vd.HashCfg(2, 4, 96, 3, 0, 0, 0), keys, None, None, ws)
     assert e.value.status == vd.ERR_INVALID_ARG
+
+
+def test_status_word_is_sticky_until_the_caller_clears_it():
+    """A device-side problem stays in the workspace's status word across later, clean calls on the same workspace."""
+    x = random_periodic(2, 4, 96, 3, seed=2)
+    bad = x.copy(); bad[0, 1, 5] = np.inf
+    cfg = vd.HashCfg(2, 4, 96, 3, 0, 0, 0)
+    keys, freqs, amp = vd.alloc_hash_outputs(cfg)
+    ws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(cfg))
+    vd.vardrop_hash(torch.from_numpy(bad).cuda(), cfg, keys, freqs, amp, ws)
+    vd.vardrop_hash(torch.from_numpy(x).cuda(), cfg, keys, freqs, amp, ws)          # a clean call does not erase the record
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.ERR_NONFINITE
+    ws[:4] = 0
+    vd.vardrop_hash(torch.from_numpy(x).cuda(), cfg, keys, freqs, amp, ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.OK
