@@ -103,9 +103,9 @@ constexpr int kBwdWorkers = 256;       // two threads per tensor-memory lane: ea
 constexpr int kBwdThreads = kBwdWorkers + 128; // plus a third warpgroup: its first warp's first lane issues every tensor-core product,
                                                // the rest of it only gives its registers to the workers
 // Register split (setmaxnreg works on whole warpgroups): the kernel is launched with 384 x 168 = 64512 registers; the
-// third warpgroup keeps 104 a thread and the two worker warpgroups take 200: 256 x 200 + 128 x 104 = 64512.
-constexpr int kBwdWorkerRegs = 200;
-constexpr int kBwdIssuerRegs = 104;
+// third warpgroup keeps 136 a thread and the two worker warpgroups take 184: 256 x 184 + 128 x 136 = 64512.
+constexpr int kBwdWorkerRegs = 184;
+constexpr int kBwdIssuerRegs = 136;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr int kQStages = 3;            // ring of query-tile operands (Q and dO), fetched two tiles ahead
 constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 2 * kQStages * kTileBytes /*Q, dO ring*/ +
@@ -281,11 +281,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 
     // operand descriptors, built once and stepped by additions: K-major views for the scores and the P^T / dS^T panels,
     // MN-major views where the reduction runs over the rows of the tile
-    const uint64_t d_k = umma_desc_sw128(smem_u32(sK), 16, 1024), d_v = umma_desc_sw128(smem_u32(sV), 16, 1024);
-    const uint64_t d_q0 = umma_desc_sw128(smem_u32(sQ), 16, 1024), d_do0 = umma_desc_sw128(smem_u32(sdO), 16, 1024);
-    const uint64_t d_pt = umma_desc_sw128(smem_u32(sPt), 16, 1024), d_dst = umma_desc_sw128(smem_u32(sdSt), 16, 1024);
-    const uint64_t m_q0 = umma_desc_sw128(smem_u32(sQ), kTileBytes, 1024), m_do0 = umma_desc_sw128(smem_u32(sdO), kTileBytes, 1024);
-    const uint64_t m_dst = umma_desc_sw128(smem_u32(sdSt), kTileBytes, 1024), m_k = umma_desc_sw128(smem_u32(sK), kTileBytes, 1024);
+    // (every tile sits at a fixed distance from the K tile, so two descriptors of the K tile and constant steps give them all)
+    const uint64_t d_k = umma_desc_sw128(smem_u32(sK), 16, 1024), m_k = umma_desc_sw128(smem_u32(sK), kTileBytes, 1024);
+    const uint64_t d_v = umma_desc_advance(d_k, kTileBytes);
+    const uint64_t d_q0 = umma_desc_advance(d_k, 2 * kTileBytes), d_do0 = umma_desc_advance(d_k, (2 + kQStages) * kTileBytes);
+    const uint64_t d_pt = umma_desc_advance(d_k, (2 + 2 * kQStages) * kTileBytes), d_dst = umma_desc_advance(d_k, (4 + 2 * kQStages) * kTileBytes);
+    const uint64_t m_q0 = umma_desc_advance(m_k, 2 * kTileBytes), m_do0 = umma_desc_advance(m_k, (2 + kQStages) * kTileBytes);
+    const uint64_t m_dst = umma_desc_advance(m_k, (4 + 2 * kQStages) * kTileBytes);
     // The five products of a (key tile, query tile) pair, each issued by one thread.  S^T = K Q^T and dP^T = V dO^T read the
     // query tile in ring stage `stage`; dV += P^T dO and dK += dS^T Q accumulate over the query loop; dQ_i = dS K.
     auto issue_st = [&](uint32_t stage) {
