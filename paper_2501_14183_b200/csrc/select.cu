@@ -363,7 +363,6 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
     int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
     const int p0 = 2 * tid, p1 = 2 * tid + 1;                     // the two items / positions this thread owns
 
-    if (s == 0 && tid == 0) *P.status = VARDROP_OK;               // nothing in this kernel can fail on the device
     uint64_t k0 = p0 < N ? keys[p0] : ~0ull, k1 = p1 < N ? keys[p1] : ~0ull;
     uint32_t n0 = p0, n1 = p1;
     bitonic_sort_regs<true>(k0, n0, k1, n1, a, idx, M);
@@ -406,15 +405,35 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
     }
     uint32_t d0 = 0, d1 = 0;
     __syncthreads();                                              // everyone is done reading the sorted keys in `a`
-    bitonic_sort_regs<false>(c0, d0, c1, d1, a, nullptr, M);
+    // Groups are usually small: a member's sampling rank is then the number of codes of its group below its own, counted over
+    // the group's few positions.  Only when some group is long does the second sort pay.
+    constexpr int kCountMaxGroup = 64;
+    const int size0 = p0 < N ? off_s[g0 + 1] - off_s[g0] : 0, size1 = p1 < N ? off_s[g1 + 1] - off_s[g1] : 0;
+    a[p0] = c0; a[p1] = c1;
+    if (!__syncthreads_or(size0 > kCountMaxGroup || size1 > kCountMaxGroup)) {
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-        const int q = 2 * tid + e;
-        const uint64_t c = e ? c1 : c0;
-        if (q < N) {
-            const int g = static_cast<int>(c >> 43), j = static_cast<int>(c & 2047u);
-            const int begin = off_s[g], size = off_s[g + 1] - begin;
-            keep_s[idx[begin + j]] = (q - begin) < quota_of(size, P.gs, P.rate_ppm);
+        for (int e = 0; e < 2; ++e) {
+            const int p = 2 * tid + e;
+            if (p < N) {
+                const uint64_t mine = e ? c1 : c0;
+                const int g = e ? g1 : g0;
+                const int begin = off_s[g], end = off_s[g + 1];
+                int below = 0;
+                for (int o = begin; o < end; ++o) below += a[o] < mine;
+                keep_s[idx[p]] = below < quota_of(end - begin, P.gs, P.rate_ppm);
+            }
+        }
+    } else {
+        bitonic_sort_regs<false>(c0, d0, c1, d1, a, nullptr, M);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int q = 2 * tid + e;
+            const uint64_t c = e ? c1 : c0;
+            if (q < N) {
+                const int g = static_cast<int>(c >> 43), j = static_cast<int>(c & 2047u);
+                const int begin = off_s[g], size = off_s[g + 1] - begin;
+                keep_s[idx[begin + j]] = (q - begin) < quota_of(size, P.gs, P.rate_ppm);
+            }
         }
     }
     __syncthreads();
