@@ -50,6 +50,16 @@ def test_select_degenerate_groups():
     check(np.full(300, 0xFFFFFFFFFFFFFFF, dtype=np.uint64), 0, 0.1, seed=3, step=9)     # 60-bit keys (k = 5)
 
 
+def test_select_group_sizes_around_the_counting_limit():
+    """The one-CTA path ranks members by counting inside groups of up to 64 and sorts when some group is longer: both sides of it."""
+    rng = np.random.default_rng(11)
+    for sizes in ([64, 64, 64], [65, 64, 64], [64, 1, 63, 2], [300, 5, 5, 5], [1] * 40 + [64]):
+        keys = np.concatenate([np.full(n, 100 + 7 * i, dtype=np.uint64) for i, n in enumerate(sizes)])
+        keys = keys[rng.permutation(len(keys))]
+        for gs, rate in ((10, 1.0), (0, 0.3)):
+            check(keys, gs, rate, seed=99, step=4)
+
+
 def test_select_multiple_scopes():
     rows = np.stack([inputs.make_keys(500, 20 + s, k=3, f_hi=25, seed=s) for s in range(5)])
     got = check(rows, 5, 1.0, seed=77, step=3)
