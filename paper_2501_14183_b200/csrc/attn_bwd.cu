@@ -166,48 +166,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                                                    const __grid_constant__ CUtensorMap map_do,
                                                                    const __grid_constant__ CUtensorMap map_acc, const BwdParams P) {
     extern __shared__ unsigned char smem_dyn[];
-    chain_wait();
-    chain_release();
-    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
-    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
-    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 100)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
-    const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
-    // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
-    // operand loads of its first work item, so the stores drain while those loads are in flight.
-    bool zeros_written = P.inv_idx == nullptr;
-    auto write_zero_rows = [&]() {
-        zeros_written = true;
-        const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
-        const int total_rows = P.B * P.N;
-        const int lane = threadIdx.x & 31;
-        const int warps_grid = gridDim.x * (kBwdWorkers >> 5);
-        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
-        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
-        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
-        int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
-        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
-        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
-            const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
-            bool dropped = false;
-            if (lane < group && r < total_rows) {
-                const int b = r / P.N, n = r - b * P.N;
-                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, dropped);
-            while (mask) {
-                const int l = __ffs(mask) - 1;
-                mask &= mask - 1;
-                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
-                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
-            }
-        }
-    };
-    if (static_cast<int>(blockIdx.x) >= n_items) {
-        if (!zeros_written && threadIdx.x < kBwdWorkers) write_zero_rows();
-        return;
-    }
-
+    // Set-up first (shared-memory carve-up, barriers, tensor memory): it touches nothing another kernel produces, so it runs
+    // while the previous kernel of the stream is still finishing.
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
     uint64_t* bar_kv = bars + 0;
     uint64_t* bar_qdo = bars + 1;                   // [3]
@@ -261,6 +221,45 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    chain_wait();
+    chain_release();
+    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
+    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 100)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
+    // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
+    // operand loads of its first work item, so the stores drain while those loads are in flight.
+    bool zeros_written = P.inv_idx == nullptr;
+    auto write_zero_rows = [&]() {
+        zeros_written = true;
+        const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
+        const int total_rows = P.B * P.N;
+        const int lane = threadIdx.x & 31;
+        const int warps_grid = gridDim.x * (kBwdWorkers >> 5);
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
+        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
+        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
+        int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
+        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
+        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
+            const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
+            bool dropped = false;
+            if (lane < group && r < total_rows) {
+                const int b = r / P.N, n = r - b * P.N;
+                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
+            }
+            unsigned mask = __ballot_sync(0xffffffffu, dropped);
+            while (mask) {
+                const int l = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
+                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
+            }
+        }
+    };
+    // (a CTA past the last item runs no loop below: it writes its share of the zero rows and frees its tensor memory)
+
     const uint32_t tm_st = tmem;            // [0,128)   S^T
     const uint32_t tm_dpt = tmem + 128;     // [128,256) dP^T
     const uint32_t tm_dv = tmem + 256;      // [256,320) dV

@@ -215,14 +215,8 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                                                                 const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v, const FwdParams P) {
     extern __shared__ unsigned char smem_dyn[];
-    chain_wait();
-    chain_release();
-    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
-    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
-    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
-    const int n_items = n_t_max * P.H * P.B;                   // work items: (query tile, head, instance); short instances skip tiles
-    if (static_cast<int>(blockIdx.x) >= n_items) return;
-
+    // Set-up first (shared-memory carve-up, barriers, tensor memory): it touches nothing another kernel produces, so it runs
+    // while the previous kernel of the stream is still finishing.
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);     // barriers and the TMEM slot sit in front of the tiles
     uint64_t* bar_q = bars + 0;
     uint64_t* bar_kv = bars + 1;                    // [2]
@@ -258,6 +252,13 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    chain_wait();
+    chain_release();
+    // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
+    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
+    const int n_items = n_t_max * P.H * P.B;                   // work items: (query tile, head, instance); short instances skip tiles
+                                                               // (a CTA past the last item falls through the loop and frees its tensor memory)
     // two 128-column buffers: S of tile j lives in buffer j & 1; once the softmax has read it, P V of the same tile
     // lands in its first 64 columns while S of tile j + 1 is produced in the other buffer
     const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
