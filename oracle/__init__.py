@@ -142,3 +142,14 @@ def rank_gaps(abar: np.ndarray, k: int) -> np.ndarray:
     amplitudes of every variate: the margin by which a variate's hash is decided."""
     top = -np.sort(-abar, axis=-1)[..., : k + 1]
     return ((top[..., :-1] - top[..., 1:]) / np.maximum(top[..., :-1], 1e-300)).min(axis=-1)
+
+
+def pearson_max(x: np.ndarray) -> np.ndarray:
+    """Appendix A, Eq. 4: for every instance and variate, the largest Pearson correlation coefficient with any other
+    variate of the same window (a constant variate correlates 0 with everything).  x [B, N, L] -> [B, N] float64."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    B, N, L = x.shape
+    out = np.empty((B, N), dtype=np.float64)
+    _load().vdo_pearson_max(_p(x), B, N, L, _p(out))
+    return out
+

@@ -354,3 +354,43 @@ void vdo_attn_bwd(const double* q, const double* k, const double* v, const doubl
         }
     }
 }
+
+/* ---------------------------------------------------------------------------------------------------
+ * Variate redundancy (Appendix A, Eq. 4): Pearson correlation coefficient between two variates of one
+ * window,  rho(v, w) = sum_i (v_i - mean v)(w_i - mean w) / (sqrt(sum_i (v_i - mean v)^2) sqrt(sum_i (w_i - mean w)^2)),
+ * and, per variate, its largest coefficient with any OTHER variate (the quantity whose histogram the
+ * appendix shows, and whose share above 0.9 Sec. 1 quotes).  The paper does not say what a constant
+ * variate gets (its denominator is zero): it is given rho = 0 with everything.
+ *   x        [B, N, L] float32
+ *   max_rho  [B, N]    for every instance: max over w != v of rho(v, w); -2 when N = 1 (no other variate)
+ * ------------------------------------------------------------------------------------------------- */
+void vdo_pearson_max(const float* x, int B, int N, int L, double* max_rho) {
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b) {
+        for (int v = 0; v < N; ++v) {
+            const float* xv = x + ((size_t)b * N + v) * L;
+            double mv = 0.0;
+            for (int i = 0; i < L; ++i) mv += (double)xv[i];
+            mv /= L;
+            double svv = 0.0;
+            for (int i = 0; i < L; ++i) svv += ((double)xv[i] - mv) * ((double)xv[i] - mv);
+            double best = -2.0;
+            for (int w = 0; w < N; ++w) {
+                if (w == v) continue;
+                const float* xw = x + ((size_t)b * N + w) * L;
+                double mw = 0.0;
+                for (int i = 0; i < L; ++i) mw += (double)xw[i];
+                mw /= L;
+                double sww = 0.0, svw = 0.0;
+                for (int i = 0; i < L; ++i) {
+                    sww += ((double)xw[i] - mw) * ((double)xw[i] - mw);
+                    svw += ((double)xv[i] - mv) * ((double)xw[i] - mw);
+                }
+                const double den = sqrt(svv) * sqrt(sww);
+                const double rho = den > 0.0 ? svw / den : 0.0;
+                if (rho > best) best = rho;
+            }
+            max_rho[(size_t)b * N + v] = best;
+        }
+    }
+}
