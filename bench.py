@@ -255,6 +255,39 @@ def kernel_table(per_kernel, work, peaks):
     return kernels
 
 
+def pearson_leg(torch, vd, path, w, peaks, barrier, args):
+    """Times vardrop_pearson_max (maximum Pearson correlation per variate, Appendix A / Eq. 4) on the workload's windows and, unless
+    --no-cpu, the oracle on one instance.  Algorithmic work: 2 B N^2 L flop (every pair once per direction)."""
+    import oracle
+    device = path.dev[0]["x"].device
+    cfg = vd.PearsonCfg(w.B, w.N, w.L, 0.9)
+    out = torch.empty((w.B, w.N), dtype=torch.float32, device=device)
+    above = torch.empty((w.B,), dtype=torch.int32, device=device)
+    ws = vd.alloc_ws(vd.vardrop_pearson_workspace_bytes(cfg), device)
+    slots = len(path.dev)
+    k = max(3, min(args.steps, 20))
+    for i in range(3):
+        vd.vardrop_pearson_max(path.dev[i % slots]["x"], cfg, out, above, ws)
+    vd.vardrop_profile_enable(True)
+    ms = time_region(torch, lambda i: vd.vardrop_pearson_max(path.dev[i % slots]["x"], cfg, out, above, ws), k, barrier)
+    per = vd.vardrop_profile_read()
+    vd.vardrop_profile_enable(False)
+    if vd.ws_status(ws) != vd.OK:
+        raise RuntimeError("device status set by vardrop_pearson_max")
+    flops = 2.0 * w.B * float(w.N) ** 2 * w.L
+    t_max = per["pearson_max_kernel"][0] / k * 1e-3
+    res = {"ms_per_call": ms / k, "normalize_us": per["pearson_normalize_kernel"][0] / k * 1e3, "max_kernel_us": t_max * 1e6,
+           "algorithmic_flops": flops, "tflops": flops / t_max / 1e12, "frac_of_bf16_peak": flops / t_max / 1e12 / peaks["bf16_tflops"],
+           "share_above_0.9": float(above.float().mean().item()) / w.N, "note": "timed with the per-kernel event timer armed"}
+    if not args.no_cpu:
+        x1 = path.host[0][0][:1].numpy()
+        t0 = time.perf_counter()
+        oracle.pearson_max(x1)
+        res["oracle_ms_per_instance"] = (time.perf_counter() - t0) * 1e3
+        res["oracle_cores"] = oracle.num_threads()
+    return res
+
+
 def run_gpu(args):
     import torch
     from paper_2501_14183_b200 import binding as vd
@@ -326,6 +359,7 @@ def run_gpu(args):
                "attn_tflops": fl / t_attn / 1e12, "attn_frac_of_bf16_peak": fl / t_attn / 1e12 / peaks["bf16_tflops"],
                "kernels": kernel_table(pk_off, kernel_work(w, w.N, selected=False), peaks),
                "note": "timed with the per-kernel event timer armed"}
+    pearson = pearson_leg(torch, vd, path, w, peaks, barrier, args) if args.pearson else None
     clocks = sampler.stop() if rank == 0 else None
     path.check_status()
 
@@ -359,6 +393,8 @@ def run_gpu(args):
                 "d2h_bytes_per_step": path.output_bytes(), "ms_per_step": ms_e2e / args.steps},
         "roofline": roofline, "kernels": kernels, "vardrop_off": off, "cpu_baseline": cpu,
     }
+    if pearson is not None:
+        line["pearson"] = pearson
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -460,6 +496,7 @@ def main():
     ap.add_argument("--impl", default="vardrop", choices=["vardrop", "reference"])
     ap.add_argument("--no-off", action="store_true", help="skip the VarDrop-off comparison pass")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline (profiling runs)")
+    ap.add_argument("--pearson", action="store_true", help="also time the variate-redundancy check (Appendix A, Eq. 4) on the workload's windows")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

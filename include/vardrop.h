@@ -214,6 +214,30 @@ int vardrop_attn_bwd(const void* q, const void* k, const void* v, const void* o,
                      const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg* cfg,
                      void* dq, void* dk, void* dv, void* ws, size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Variate redundancy -- Appendix A ("Variate Redundancy in Multivariate Time Series Benchmark Datasets"),
+ * Eq. 4: the Pearson correlation coefficient rho(v, w) of two variates of one window, and per variate
+ * its largest coefficient with any other variate (the quantity of the appendix's histograms; Sec. 1
+ * quotes the share of variates above 0.9).  A constant variate (zero variance; the paper leaves it
+ * undefined) correlates 0 with everything.
+ *
+ * x          [B, N, L] float32, contiguous, device: every instance is treated on its own.
+ * max_rho    [B, N] float32, device: max over w != v of rho(v, w); -2 when N = 1.
+ * n_above    [B] int32, device: number of variates of the instance with max_rho >= cfg->threshold.
+ * ws         scratch (status word + the normalised windows); vardrop_pearson_workspace_bytes.
+ * Accuracy: statistics in fp32, the products on the tensor cores with every value held as two bf16
+ * terms (16 mantissa bits) and fp32 accumulation: absolute error of a coefficient below 1e-4.
+ * Device status: VARDROP_ERR_NONFINITE when a window's variance is not finite.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t B, N, L;
+    float threshold;     /* in [-1, 1] */
+} vardrop_pearson_cfg;
+
+size_t vardrop_pearson_workspace_bytes(const vardrop_pearson_cfg* cfg);
+int vardrop_pearson_max(const float* x, const vardrop_pearson_cfg* cfg, float* max_rho, int32_t* n_above, void* ws,
+                        size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -33,6 +33,10 @@ class AttnCfg(C.Structure):
     _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float), ("S", C.c_int32)]
 
 
+class PearsonCfg(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("L", C.c_int32), ("threshold", C.c_float)]
+
+
 class VardropError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -42,7 +46,7 @@ class VardropError(RuntimeError):
 
 EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_hash_workspace_bytes", "vardrop_hash",
            "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_select_static", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
-           "vardrop_attn_bwd", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
+           "vardrop_attn_bwd", "vardrop_pearson_workspace_bytes", "vardrop_pearson_max", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
            "vardrop_profile_kernel_name", "vardrop_profile_read")
 
 
@@ -56,7 +60,8 @@ def load() -> C.CDLL:
         for name in ("vardrop_status_string", "vardrop_last_error", "vardrop_version"):
             getattr(lib, name).restype = C.c_char_p
         lib.vardrop_status_string.argtypes = [C.c_int]
-        for name in ("vardrop_hash_workspace_bytes", "vardrop_select_workspace_bytes", "vardrop_attn_workspace_bytes"):
+        for name in ("vardrop_hash_workspace_bytes", "vardrop_select_workspace_bytes", "vardrop_attn_workspace_bytes",
+                     "vardrop_pearson_workspace_bytes"):
             getattr(lib, name).restype = C.c_size_t
             getattr(lib, name).argtypes = [C.c_void_p]
         lib.vardrop_hash.restype = C.c_int
@@ -69,6 +74,8 @@ def load() -> C.CDLL:
         lib.vardrop_attn_fwd.argtypes = [C.c_void_p] * 9 + [C.c_size_t, C.c_void_p]
         lib.vardrop_attn_bwd.restype = C.c_int
         lib.vardrop_attn_bwd.argtypes = [C.c_void_p] * 14 + [C.c_size_t, C.c_void_p]
+        lib.vardrop_pearson_max.restype = C.c_int
+        lib.vardrop_pearson_max.argtypes = [C.c_void_p] * 5 + [C.c_size_t, C.c_void_p]
         lib.vardrop_launch_count.restype = C.c_longlong
         lib.vardrop_profile_kernel_name.restype = C.c_char_p
         lib.vardrop_profile_kernel_name.argtypes = [C.c_int]
@@ -139,6 +146,15 @@ def vardrop_attn_bwd(q, k, v, o, lse, d_o, sel_idx, n_sel, inv_idx, cfg: AttnCfg
     _check(load().vardrop_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(sel_idx), _ptr(n_sel),
                                    _ptr(inv_idx), C.byref(cfg), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws),
                                    ws.numel() * ws.element_size(), _stream()), "vardrop_attn_bwd")
+
+
+def vardrop_pearson_workspace_bytes(cfg: PearsonCfg) -> int:
+    return int(load().vardrop_pearson_workspace_bytes(C.byref(cfg)))
+
+
+def vardrop_pearson_max(x, cfg: PearsonCfg, max_rho, n_above, ws) -> None:
+    _check(load().vardrop_pearson_max(_ptr(x), C.byref(cfg), _ptr(max_rho), _ptr(n_above), _ptr(ws), ws.numel() * ws.element_size(),
+                                      _stream()), "vardrop_pearson_max")
 
 
 def vardrop_launch_count() -> int:

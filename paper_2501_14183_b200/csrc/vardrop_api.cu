@@ -47,7 +47,8 @@ long long g_launches = 0;
 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_events[K_COUNT];   // pairs recorded since the timer was armed
 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_free;              // pairs ready for reuse
 const char* const g_kernel_names[K_COUNT] = {"hash_kernel", "select_small_kernel", "select_count_kernel", "select_group_kernel", "select_sample_kernel", "gather_kernel",
-                                             "attn_fwd_kernel", "bwd_prep_kernel", "attn_bwd_kernel", "bwd_convert_kernel"};
+                                             "attn_fwd_kernel", "bwd_prep_kernel", "attn_bwd_kernel", "bwd_convert_kernel", "pearson_normalize_kernel",
+                                             "pearson_max_kernel"};
 }  // namespace
 
 LaunchScope::LaunchScope(int id, cudaStream_t stream) : id_(id), stream_(stream), stop_(nullptr) {
@@ -224,6 +225,22 @@ int vardrop_attn_bwd(const void* q, const void* k, const void* v, const void* o,
     VD_CHECK(check_ptr(dv, "dv", true));
     VD_CHECK(check_ws(ws, ws_bytes, attn_workspace_bytes(*cfg)));
     return attn_bwd_launch(q, k, v, o, lse, d_o, sel_idx, n_sel, inv_idx, *cfg, dq, dk, dv, ws, static_cast<cudaStream_t>(stream));
+}
+
+size_t vardrop_pearson_workspace_bytes(const vardrop_pearson_cfg* cfg) {
+    if (!cfg || pearson_validate(*cfg) != VARDROP_OK) return 0;
+    return pearson_workspace_bytes(*cfg);
+}
+
+int vardrop_pearson_max(const float* x, const vardrop_pearson_cfg* cfg, float* max_rho, int32_t* n_above, void* ws, size_t ws_bytes,
+                        void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(pearson_validate(*cfg));
+    VD_CHECK(check_ptr(x, "x", true));
+    VD_CHECK(check_ptr(max_rho, "max_rho", true));
+    VD_CHECK(check_ptr(n_above, "n_above", true));
+    VD_CHECK(check_ws(ws, ws_bytes, pearson_workspace_bytes(*cfg)));
+    return pearson_launch(x, *cfg, max_rho, n_above, ws, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
