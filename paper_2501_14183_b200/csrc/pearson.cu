@@ -5,10 +5,11 @@
 //
 // pearson_normalize_kernel   one warp per (instance, variate): mean and centred norm in fp32, then the unit vector
 //                            z = (x - mean) / |x - mean| is stored as two bf16 terms, z = hi + lo (16 mantissa bits),
-//                            in [B, Npad, Lpad] arrays padded with zeros (Npad a multiple of 128, Lpad of 64).
-// pearson_max_kernel         one CTA per (128-variate row tile, instance) walks over the column tiles: rho = z_v . z_w is a
-//                            dense contraction, so it runs on the tcgen05 tensor cores (hi hi + hi lo + lo hi, fp32
-//                            accumulator in tensor memory); one thread per row takes the maximum over the other variates.
+//                            in [B, Npad, Lpad] arrays padded with zeros (Npad a multiple of 256, Lpad of 64).
+// pearson_max_kernel         one CTA per (128-variate row tile, instance) walks over 256-variate column tiles: rho = z_v . z_w is
+//                            a dense contraction, so it runs on the tcgen05 tensor cores (hi hi + hi lo + lo hi, fp32
+//                            accumulator in tensor memory); operand chunks are fetched into registers one step ahead of
+//                            the products; two threads per row take the maximum over the other variates.
 #include "attn_common.cuh"
 
 namespace vardrop {
@@ -61,19 +62,20 @@ __global__ void __launch_bounds__(256) pearson_normalize_kernel(const PearsonPar
     }
 }
 
-constexpr int kPearsonThreads = 128;
-constexpr int kPearsonSmemBytes = 1024 /*barrier, alignment*/ + 4 * kTileBytes /*row tile hi, lo; column tile hi, lo*/;
-constexpr uint32_t kPearsonTmemCols = 128;
+constexpr int kPearsonThreads = 256;                 // two threads per row: each takes 128 of the 256 columns of a step
+constexpr int kColTile = 256;                        // column variates per step (one N = 256 product)
+constexpr int kPearsonSmemBytes = 1024 /*barrier, row maxima, alignment*/ + 2 * kTileBytes /*row tile hi, lo*/ + 4 * kTileBytes /*column tile hi, lo*/;
+constexpr uint32_t kPearsonTmemCols = 256;
+constexpr int kPearsonChunks = (2 * 1024 + 2 * 2048) / kPearsonThreads;      // 16-byte chunks a thread moves per step (24)
 
 __global__ void __launch_bounds__(kPearsonThreads) pearson_max_kernel(const PearsonParams P) {
     extern __shared__ unsigned char smem_dyn[];
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem_dyn);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 8);
-    unsigned char* sA_hi = align_tiles(smem_dyn + 16);
-    unsigned char* sA_lo = sA_hi + kTileBytes;
-    unsigned char* sB_hi = sA_lo + kTileBytes;
-    unsigned char* sB_lo = sB_hi + kTileBytes;
-    if (sB_lo + kTileBytes > smem_dyn + kPearsonSmemBytes) {     // dynamic shared memory base not 1024-byte aligned
+    float* s_best = reinterpret_cast<float*>(smem_dyn + 64);     // [128] maxima of the threads that take columns 128 .. 255
+    unsigned char* sA = align_tiles(smem_dyn + 64 + kTile * sizeof(float));      // row tile: hi, then lo (16 KB each)
+    unsigned char* sB = sA + 2 * kTileBytes;                                     // column tile: hi, then lo (32 KB each)
+    if (sB + 4 * kTileBytes > smem_dyn + kPearsonSmemBytes) {    // dynamic shared memory base not 1024-byte aligned
         if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
         return;
     }
@@ -94,85 +96,103 @@ __global__ void __launch_bounds__(kPearsonThreads) pearson_max_kernel(const Pear
     chain_release();
 
     const int b = blockIdx.y, ti = blockIdx.x;
-    const int n_tiles = P.Npad / kTile, n_chunks = P.Lpad / 64;
+    const int n_col_tiles = P.Npad / kColTile, n_chunks = P.Lpad / 64, n_steps = n_col_tiles * n_chunks;
     const int chunks_row = P.Lpad / 8;                           // 16-byte chunks per stored row
     const uint4* zh = reinterpret_cast<const uint4*>(P.z_hi) + static_cast<size_t>(b) * P.Npad * chunks_row;
     const uint4* zl = reinterpret_cast<const uint4*>(P.z_lo) + static_cast<size_t>(b) * P.Npad * chunks_row;
-    constexpr uint32_t idesc = umma_idesc_bf16(128, 128, 0, 0);
-    const uint64_t d_ah = umma_desc_sw128(smem_u32(sA_hi), 16, 1024);
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
-    const int v = ti * kTile + tid;                              // this thread's variate
+    constexpr uint32_t idesc = umma_idesc_bf16(128, kColTile, 0, 0);
+    const uint64_t d_ah = umma_desc_sw128(smem_u32(sA), 16, 1024);
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int row = tid & (kTile - 1), chalf = tid >> 7;         // tensor-memory lane and which 128 columns of it
+    const int v = ti * kTile + row;                              // this thread's variate
     float best = -2.f;
     uint32_t phase = 0;
-    bool ok = true;
+    bool ok = true, pending = false;
 
-    for (int tj = 0; tj < n_tiles && ok; ++tj) {
-        for (int kc = 0; kc < n_chunks; ++kc) {
-            // the four 128 x 64 tiles of this step, 16-byte chunks spread over the CTA, stored with the 128-byte swizzle
+    // A step = 64 time steps of one column tile: the row tile's and the column tile's hi / lo chunks, 24 per thread.  They are
+    // fetched into registers one step ahead, while the previous step's products run, and parked in shared memory (128-byte
+    // swizzle) once those products are done.
+    uint4 regs[kPearsonChunks];
+    auto fetch = [&](int step) {
+        const int tj = step / n_chunks, kc = step - tj * n_chunks;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint4 va[4], vb[4], vc[4], vd[4];
+        for (int u = 0; u < kPearsonChunks; ++u) {
+            const int idx = tid + kPearsonThreads * u;           // 0 .. 6143: A hi, A lo (1024 each), B hi, B lo (2048 each)
+            const bool is_a = idx < 2048;
+            const int local = is_a ? (idx & 1023) : ((idx - 2048) & 2047);
+            const bool lo_half = is_a ? idx >= 1024 : idx >= 4096;
+            const int r = local >> 3, ch = local & 7;
+            const size_t o = static_cast<size_t>((is_a ? ti * kTile : tj * kColTile) + r) * chunks_row + kc * 8 + ch;
+            regs[u] = __ldg((lo_half ? zl : zh) + o);
+        }
+    };
+    auto park = [&]() {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int idx = tid + kPearsonThreads * (4 * half + u);
-                    const int r = idx >> 3, ch = idx & 7;
-                    const size_t oa = static_cast<size_t>(ti * kTile + r) * chunks_row + kc * 8 + ch;
-                    const size_t ob = static_cast<size_t>(tj * kTile + r) * chunks_row + kc * 8 + ch;
-                    va[u] = __ldg(zh + oa);
-                    vb[u] = __ldg(zl + oa);
-                    vc[u] = __ldg(zh + ob);
-                    vd[u] = __ldg(zl + ob);
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int idx = tid + kPearsonThreads * (4 * half + u);
-                    const int r = idx >> 3, ch = idx & 7;
-                    const int off = r * kRowBytes + ((ch ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(sA_hi + off) = va[u];
-                    *reinterpret_cast<uint4*>(sA_lo + off) = vb[u];
-                    *reinterpret_cast<uint4*>(sB_hi + off) = vc[u];
-                    *reinterpret_cast<uint4*>(sB_lo + off) = vd[u];
-                }
-            }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {                                      // rho += hi hi + hi lo + lo hi over these 64 time steps
-                tc_fence_after();
-                const uint64_t d_al = umma_desc_advance(d_ah, kTileBytes), d_bh = umma_desc_advance(d_ah, 2 * kTileBytes);
-                const uint64_t d_bl = umma_desc_advance(d_ah, 3 * kTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    tc_mma_bf16(tmem, umma_desc_advance(d_ah, ks * 32), umma_desc_advance(d_bh, ks * 32), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
-                    tc_mma_bf16(tmem, umma_desc_advance(d_ah, ks * 32), umma_desc_advance(d_bl, ks * 32), idesc, 1u);
-                    tc_mma_bf16(tmem, umma_desc_advance(d_al, ks * 32), umma_desc_advance(d_bh, ks * 32), idesc, 1u);
-                }
-                tc_commit(bar);
-            }
-            ok &= mbar_wait(bar, phase);                         // products done: the tiles may be overwritten
+        for (int u = 0; u < kPearsonChunks; ++u) {
+            const int idx = tid + kPearsonThreads * u;
+            const bool is_a = idx < 2048;
+            const int local = is_a ? (idx & 1023) : ((idx - 2048) & 2047);
+            const bool lo_half = is_a ? idx >= 1024 : idx >= 4096;
+            const int r = local >> 3, ch = local & 7;
+            unsigned char* tile = is_a ? sA + (lo_half ? kTileBytes : 0) : sB + (lo_half ? 2 * kTileBytes : 0);
+            *reinterpret_cast<uint4*>(tile + r * kRowBytes + ((ch ^ (r & 7)) << 4)) = regs[u];
+        }
+    };
+
+    if (n_steps > 0) fetch(0);
+    for (int step = 0; step < n_steps && ok; ++step) {
+        const int tj = step / n_chunks, kc = step - tj * n_chunks;
+        if (pending) {                                           // the previous step's products are done: its tiles may be overwritten
+            ok &= mbar_wait(bar, phase);
             phase ^= 1u;
-            ok = __syncthreads_and(ok);
-            if (!ok) break;
+            pending = false;
         }
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            float r[32];
-            tmem_ld32(tmem + lane_sel + c * 32, r);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int w = tj * kTile + c * 32 + i;
-                if (w < P.N && w != v) best = fmaxf(best, r[i]);
-            }
-        }
+        park();
+        fence_proxy_async_smem();
         tc_fence_before();
-        __syncthreads();                                         // every row is read before the next column tile's products
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        if (tid == 0) {                                          // rho += hi hi + hi lo + lo hi over these 64 time steps
+            tc_fence_after();
+            const uint64_t d_al = umma_desc_advance(d_ah, kTileBytes), d_bh = umma_desc_advance(d_ah, 2 * kTileBytes);
+            const uint64_t d_bl = umma_desc_advance(d_ah, 4 * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                tc_mma_bf16(tmem, umma_desc_advance(d_ah, ks * 32), umma_desc_advance(d_bh, ks * 32), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
+                tc_mma_bf16(tmem, umma_desc_advance(d_ah, ks * 32), umma_desc_advance(d_bl, ks * 32), idesc, 1u);
+                tc_mma_bf16(tmem, umma_desc_advance(d_al, ks * 32), umma_desc_advance(d_bh, ks * 32), idesc, 1u);
+            }
+            tc_commit(bar);
+        }
+        pending = true;
+        if (step + 1 < n_steps) fetch(step + 1);                 // in flight while the products run
+        if (kc + 1 == n_chunks) {                                // the column tile is complete: this thread's row, its 128 columns
+            ok &= mbar_wait(bar, phase);
+            phase ^= 1u;
+            pending = false;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float r[32];
+                tmem_ld32(tmem + lane_sel + chalf * 128 + c * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int w = tj * kColTile + chalf * 128 + c * 32 + i;
+                    if (w < P.N && w != v) best = fmaxf(best, r[i]);
+                }
+            }
+            tc_fence_before();
+            ok = __syncthreads_and(ok);                          // every row is read before the next column tile's products
+        }
     }
 
-    if (ok && v < P.N) P.max_rho[static_cast<size_t>(b) * P.N + v] = best;
-    const unsigned above = __ballot_sync(0xffffffffu, ok && v < P.N && best >= P.threshold);
+    if (chalf == 1) s_best[row] = best;
+    __syncthreads();
+    if (chalf == 0) best = fmaxf(best, s_best[row]);
+    const bool mine = chalf == 0 && ok && v < P.N;
+    if (mine) P.max_rho[static_cast<size_t>(b) * P.N + v] = best;
+    const unsigned above = __ballot_sync(0xffffffffu, mine && best >= P.threshold);
     if ((tid & 31) == 0 && above) atomicAdd(P.n_above + b, __popc(above));
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     tc_fence_before();
@@ -186,7 +206,7 @@ struct PearsonWs {
 };
 PearsonWs pearson_layout(const vardrop_pearson_cfg& c) {
     PearsonWs w;
-    w.Npad = (c.N + kTile - 1) / kTile * kTile;
+    w.Npad = (c.N + kColTile - 1) / kColTile * kColTile;
     w.Lpad = (c.L + 63) / 64 * 64;
     const size_t bytes = align_up(static_cast<size_t>(c.B) * w.Npad * w.Lpad * sizeof(__nv_bfloat16), 1024);
     w.z_hi = kWsHeaderBytes;
@@ -224,7 +244,7 @@ int pearson_launch(const float* x, const vardrop_pearson_cfg& c, float* max_rho,
         if (int st = check_cuda(cudaFuncSetAttribute(pearson_max_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPearsonSmemBytes), "pearson: smem attribute")) return st;
         attr_dev = dev;
     }
-    { LaunchScope ls_(K_PEARSON_MAX, stream); err = launch_chained(pearson_max_kernel, dim3(w.Npad / kTile, c.B), dim3(kPearsonThreads), kPearsonSmemBytes, stream, P); }
+    { LaunchScope ls_(K_PEARSON_MAX, stream); err = launch_chained(pearson_max_kernel, dim3((c.N + kTile - 1) / kTile, c.B), dim3(kPearsonThreads), kPearsonSmemBytes, stream, P); }
     return check_cuda(err, "pearson: launch");
 }
 
