@@ -68,7 +68,7 @@ constexpr int kPearsonSmemBytes = 1024 /*barrier, row maxima, alignment*/ + 2 * 
 constexpr uint32_t kPearsonTmemCols = 256;
 constexpr int kPearsonChunks = (2 * 1024 + 2 * 2048) / kPearsonThreads;      // 16-byte chunks a thread moves per step (24)
 
-__global__ void __launch_bounds__(kPearsonThreads) pearson_max_kernel(const PearsonParams P) {
+__global__ void __launch_bounds__(kPearsonThreads, 2) pearson_max_kernel(const PearsonParams P) {
     extern __shared__ unsigned char smem_dyn[];
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem_dyn);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 8);
