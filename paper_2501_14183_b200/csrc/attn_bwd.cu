@@ -180,7 +180,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint64_t* bar_conv = bars + 10;                 // the "last key tile of its (instance, head)" flag of an item is written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 96);
     float* s_stat = reinterpret_cast<float*>(smem_dyn + 128);     // [3 stages][128] lse of the query tile, log2 domain
-    float* s_dpart = s_stat + kQStages * kTile;                   // [2 halves][128] partial Delta = sum over 32 head dims of dO O
+    float* s_dpart = s_stat + kQStages * kTile;                   // [2][128] Delta of the query tile: with precomputed Delta, one array per
+                                                                  // tile parity (written a barrier ahead of its use); otherwise the two
+                                                                  // halves' partial sums over 32 head dimensions of dO O
     unsigned char* sK = align_tiles(smem_dyn + 128 + (kQStages + 2) * kTile * sizeof(float));
     unsigned char* sV = sK + kTileBytes;
     unsigned char* sQ = sV + kTileBytes;            // 3 stages
@@ -480,6 +482,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             s_stat[st0 * kTile + row] = lse_first;
             if (n_q > 1) s_stat[((st0 + 1) % kQStages) * kTile + row] = lse_second;
         }
+        if (use_delta && half == 1) s_dpart[(q_count & 1) * kTile + row] = dl_cur;      // Delta of the first tile, in its parity's array
         if (!zeros_written) write_zero_rows();
         worker_sync();                                   // row statistics of the first tiles visible
 
@@ -496,9 +499,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 dl_next = load_delta(b, h, (i + 1) * kTile + row);
                 if (!use_delta) load_o(b, h, (i + 1) * kTile + row, o_next);
             }
-            if (use_delta) {
-                if (half == 1) s_dpart[row] = dl_cur;    // the complete value: phase B reads one array
-            } else {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
+            if (!use_delta) {   // Delta of query `row`, this thread's 32 head dimensions: dO from the tile in shared memory, O from registers
                 ok &= mbar_wait(bar_qdo + st, (q_count / kQStages) & 1);
                 const unsigned char* do_row = sdO + st * kTileBytes + row * kRowBytes;
                 float part = 0.f;
@@ -506,6 +507,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 for (int x = 0; x < 4; ++x)
                     part += dot8(o_cur[x], *reinterpret_cast<const uint4*>(do_row + (((half * 4 + x) ^ (row & 7)) << 4)));
                 s_dpart[half * kTile + row] = part;
+                worker_sync();                           // every partial sum is in place before phase B reads them
             }
 
             // ---- phase A: P^T of this thread's key row, its 64 queries (kept in registers for phase B) ----------
@@ -540,7 +542,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             tc_fence_after();
             if (i + 2 < n_q) fetch_qdo(i + 2, st2);
             {
-                const float* dlt = s_dpart + half * 64;
+                const float* dlt = s_dpart + (use_delta ? (q_count & 1) * kTile : 0) + half * 64;
                 float dp[2][16];
                 tmem_ld16(tm_dpt + lane_sel + half * 64, dp[0]);
 #pragma unroll
@@ -573,6 +575,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             }
             if (i + 2 < n_q && half == 0) s_stat[st2 * kTile + row] = lse_ahead;       // read two tiles from now, behind several barriers
             if (i + 1 < n_q) {
+                // precomputed Delta of the next tile goes into the other parity's array now: the barrier at the end of this
+                // iteration stands between this store and its readers, and that array's last readers are a barrier behind
+                if (use_delta && half == 1) s_dpart[((q_count + 1) & 1) * kTile + row] = dl_next;
                 dl_cur = dl_next;
                 if (!use_delta) {
 #pragma unroll

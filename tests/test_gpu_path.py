@@ -129,3 +129,56 @@ def test_whole_path_per_instance_scope():
         assert_attn_close(dq[b:b + 1].double().cpu().numpy(), wq, f"dq[{b}]")
         assert_attn_close(dk[b:b + 1].double().cpu().numpy(), wk, f"dk[{b}]")
         assert_attn_close(dv[b:b + 1].double().cpu().numpy(), wv, f"dv[{b}]")
+
+
+@pytest.mark.parametrize("name", ["elec", "traffic"])
+def test_back_to_back_steps_match_isolated_steps(name):
+    """Steps queued without any synchronisation (kernels chained by programmatic dependent launches, shared workspaces and
+    selection buffers reused from step to step) give bit for bit what the same steps give when the device is synchronised
+    after every call."""
+    import bench
+    w = inputs.WORKLOADS[name]
+    device = torch.device("cuda", 0)
+    names = ("o", "lse", "dq", "dk", "dv")
+
+    def run(sync_each_call):
+        path = bench.Path(w, device, seed=w.seed, slots=3)
+        for d in path.dev:
+            for n in ("dq", "dk", "dv"):
+                d[n].fill_(float("nan"))
+        if sync_each_call:
+            real = {}
+            for fn in ("vardrop_hash", "vardrop_select", "vardrop_attn_fwd", "vardrop_attn_bwd"):
+                real[fn] = getattr(vd, fn)
+
+                def wrapped(*a, _f=real[fn]):
+                    _f(*a)
+                    torch.cuda.synchronize()
+                setattr(vd, fn, wrapped)
+        try:
+            torch.cuda.synchronize()
+            for s in range(3):
+                path.step(s)
+        finally:
+            if sync_each_call:
+                for fn, f in real.items():
+                    setattr(vd, fn, f)
+        torch.cuda.synchronize()
+        path.check_status()
+        return [{n: path.dev[s][n].clone() for n in names} for s in range(3)], int(path.sel["n_sel"].item())
+
+    chained, kept = run(False)
+    isolated, kept_i = run(True)
+    assert kept == kept_i
+    for s in range(3):
+        for n in names:
+            a, b = chained[s][n], isolated[s][n]
+            if n == "o":
+                a, b = a[:, :kept], b[:, :kept]
+            elif n == "lse":
+                a, b = a[:, :, :kept], b[:, :, :kept]
+            if not torch.equal(a.view(torch.uint8), b.view(torch.uint8)):
+                diff = (a.float() - b.float()).abs()
+                diff = torch.nan_to_num(diff, nan=1e9)
+                raise AssertionError(f"step {s} tensor {n}: {int((diff > 0).sum())} differing elements, max {float(diff.max()):.3e}, "
+                                     f"first at {torch.nonzero(diff > 0)[0].tolist()}")
