@@ -1,14 +1,16 @@
-// Grouping by hash value and stratified sampling (Eq. 1, Eq. 2) in two launches, without a sort and
-// without any spin-wait.
+// Grouping by hash value and stratified sampling (Eq. 1, Eq. 2), without a spin-wait.
 //
-// Launch 1 (count + finish-by-last-CTA): every CTA compares a slice of variates against a slice of keys
-// and adds, per variate n, lt[n] = #{m : key_m < key_n} and eq[n] = #{m < n : key_m = key_n} with integer
-// atomics.  lt[n] is the start of n's group in (key, index) order and eq[n] is n's rank inside its group,
-// so lt + eq is n's sorted position.  The CTA that finishes last for a hash row scatters the members,
-// scans the group heads into dense group ids / offsets, and draws each member's Philox priority.
-// Launch 2 (rank in group + finish-by-last-CTA): every member counts the members of its own group with a
-// smaller (priority, rank) pair; it is kept when that count is below the group's quota.  The last CTA of a
-// hash row compacts the kept variates into sel_idx / inv_idx with one scan.
+// Small problems (N <= 2048): one CTA per hash row does everything in shared memory (select_small_kernel).
+// Larger ones take three launches:
+//   select_count_kernel   every CTA compares a slice of variates against a slice of keys and adds, per variate n,
+//                         lt[n] = #{m : key_m < key_n} and eq[n] = #{m < n : key_m = key_n} with integer atomics.  lt[n] is
+//                         the start of n's group in (key, index) order and eq[n] is n's rank inside its group, so lt + eq
+//                         is n's sorted position.
+//   select_group_kernel   one CTA per hash row scatters the members, scans the group heads into dense group ids and
+//                         offsets, and draws each member's Philox priority.
+//   select_sample_kernel  every member counts the members of its own group with a smaller (priority, rank) pair; it is
+//                         kept when that count is below the group's quota.  The CTA that finishes last for a hash row
+//                         compacts the kept variates into sel_idx / inv_idx with one scan.
 #include <mutex>
 
 #include "common.cuh"
@@ -18,8 +20,12 @@ namespace vardrop {
 
 namespace {
 
-constexpr int kSelThreads = 256;
-constexpr int kKeyChunk = 128;     // keys compared per CTA in launch 1
+constexpr int kSelThreads = 256;    // select_count_kernel
+constexpr int kTailThreads = 1024;  // select_group_kernel, select_sample_kernel: one CTA walks a whole hash row, so the
+                                    // round trips to memory are spread over as many threads as a CTA can have
+constexpr int kTailChunks = 8;      // positions per thread in a batch of the ordered compaction (64 registers a thread)
+constexpr int kKeyChunk = 128;      // keys compared per CTA by select_count_kernel
+constexpr size_t kGroupMaxSmem = 216 * 1024;   // select_group_kernel keeps 12 bytes per variate in shared memory up to this
 
 struct SelectParams {
     const uint64_t* keys;
@@ -61,8 +67,9 @@ __device__ __forceinline__ int quota_of(int size, int gs, long long rate_ppm) {
     return static_cast<int>(q);
 }
 
-// Inclusive scan of one int per thread across the CTA (kSelThreads threads); returns this thread's inclusive value
+// Inclusive scan of one int per thread across the CTA (kThreads threads); returns this thread's inclusive value
 // and the CTA total through `total`.
+template <int kThreads>
 __device__ __forceinline__ int block_scan_inclusive(int v, int* warp_sums, int* total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -75,7 +82,7 @@ __device__ __forceinline__ int block_scan_inclusive(int v, int* warp_sums, int* 
     __syncthreads();
     int base = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kSelThreads / 32; ++w) {
+    for (int w = 0; w < kThreads / 32; ++w) {
         const int s = warp_sums[w];
         if (w < warp) base += s;
         tot += s;
@@ -98,46 +105,48 @@ __device__ __forceinline__ bool last_cta_of_row(unsigned int* counter, unsigned 
     return last;
 }
 
-// Ordered compaction by one CTA: for every position p < N, in ascending order, `emit(p, set, before, payload)` is called
-// with (set, payload) = flag(p) and before = number of set flags at positions below p; returns the number of set flags.
-// Positions are dealt to the threads round-robin (position = batch base + chunk * kSelThreads + thread) and a batch of 32
-// chunks is handled with fully unrolled loops, so the (dependent) loads behind the 32 flags of a thread are coalesced and
-// all in flight at once instead of one memory round trip per position; a batch is ordered with warp ballots and one scan of
-// the per-warp counts.
-template <class FlagFn, class EmitFn>
+// Ordered compaction by one CTA of kThreads threads: for every position p < N, in ascending order,
+// `emit(p, set, before, payload)` is called with (set, payload) = flag(p) and before = number of set flags at positions
+// below p; returns the number of set flags.  Positions are dealt to the threads round-robin (position = batch base +
+// chunk * kThreads + thread) and a batch of kChunks chunks is handled with fully unrolled loops, so the (dependent) loads
+// behind the flags of a thread are coalesced and all in flight at once instead of one memory round trip per position; a
+// batch is ordered with warp ballots and one scan of the per-warp counts.
+template <int kThreads, int kChunks, class FlagFn, class EmitFn>
 __device__ __forceinline__ int ordered_compact(int N, FlagFn flag, EmitFn emit) {
-    constexpr int kWarps = kSelThreads / 32;
-    __shared__ uint32_t s_mask[32 * kWarps];      // ballot of chunk k, warp w at [k * kWarps + w]: position order
-    __shared__ int s_excl[32 * kWarps];           // set flags of the batch before that (chunk, warp)
+    constexpr int kWarps = kThreads / 32;
+    static_assert(kChunks <= 32 && kChunks * kWarps <= kThreads, "one ballot word per thread at most");
+    __shared__ uint32_t s_mask[kChunks * kWarps];  // ballot of chunk k, warp w at [k * kWarps + w]: position order
+    __shared__ int s_excl[kChunks * kWarps];       // set flags of the batch before that (chunk, warp)
     __shared__ int s_warp[kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int done = 0;                                  // set flags of the batches before this one
-    for (int base = 0; base < N; base += 32 * kSelThreads) {
-        uint32_t bits = 0;                         // bit k: flag of position base + k * kSelThreads + thread
-        int payload[32];
+    for (int base = 0; base < N; base += kChunks * kThreads) {
+        uint32_t bits = 0;                         // bit k: flag of position base + k * kThreads + thread
+        int payload[kChunks];
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-            const int p = base + k * kSelThreads + static_cast<int>(threadIdx.x);
+        for (int k = 0; k < kChunks; ++k) {
+            const int p = base + k * kThreads + static_cast<int>(threadIdx.x);
             payload[k] = 0;
             if (p < N && flag(p, &payload[k])) bits |= 1u << k;
         }
         uint32_t mine = 0;
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
+        for (int k = 0; k < kChunks; ++k) {
             const uint32_t m = __ballot_sync(0xffffffffu, (bits >> k) & 1u);
             if (lane == k) mine = m;
         }
         __syncthreads();                           // the tables of the previous batch are no longer read
-        s_mask[lane * kWarps + warp] = mine;
+        if (lane < kChunks) s_mask[lane * kWarps + warp] = mine;
         __syncthreads();
         int total = 0;
-        const int cnt = __popc(s_mask[threadIdx.x]);               // kSelThreads = 32 * kWarps entries, one per thread
-        const int incl = block_scan_inclusive(cnt, s_warp, &total);
-        s_excl[threadIdx.x] = incl - cnt;
+        const bool entry = static_cast<int>(threadIdx.x) < kChunks * kWarps;      // one (chunk, warp) ballot per thread
+        const int cnt = entry ? __popc(s_mask[threadIdx.x]) : 0;
+        const int incl = block_scan_inclusive<kThreads>(cnt, s_warp, &total);
+        if (entry) s_excl[threadIdx.x] = incl - cnt;
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-            const int p = base + k * kSelThreads + static_cast<int>(threadIdx.x);
+        for (int k = 0; k < kChunks; ++k) {
+            const int p = base + k * kThreads + static_cast<int>(threadIdx.x);
             if (p < N) {
                 const uint32_t m = s_mask[k * kWarps + warp];
                 emit(p, ((bits >> k) & 1u) != 0, done + s_excl[k * kWarps + warp] + __popc(m & ((1u << lane) - 1u)), payload[k]);
@@ -164,10 +173,21 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectP
     if (n < N) {
         const uint64_t mine = keys[n];
         int c_lt = 0, c_eq = 0;
-        for (int i = 0; i < mcount; ++i) {
-            const uint64_t other = skeys[i];
-            c_lt += other < mine;
-            c_eq += (other == mine) & (m0 + i < n);
+        const int n_first = blockIdx.x * kSelThreads;
+        if (m0 >= n_first + kSelThreads) {                 // every key of the slice has a higher index than every variate here
+            for (int i = 0; i < mcount; ++i) c_lt += skeys[i] < mine;
+        } else if (m0 + mcount <= n_first) {               // every key of the slice has a lower index
+            for (int i = 0; i < mcount; ++i) {
+                const uint64_t other = skeys[i];
+                c_lt += other < mine;
+                c_eq += other == mine;
+            }
+        } else {
+            for (int i = 0; i < mcount; ++i) {
+                const uint64_t other = skeys[i];
+                c_lt += other < mine;
+                c_eq += (other == mine) & (m0 + i < n);
+            }
         }
         if (c_lt) atomicAdd(lt + n, c_lt);
         if (c_eq) atomicAdd(eq + n, c_eq);
@@ -175,55 +195,73 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(const SelectP
 }
 
 // One CTA per hash row, after the counts are complete: members, group heads -> ids and offsets, priorities.
-__global__ void __launch_bounds__(kSelThreads) select_group_kernel(const SelectParams P) {
+// The three passes reach members / eq / group ids through the sorted positions, i.e. in scattered order.  A single SM
+// turns every scattered warp access to global memory into 32 separate requests, which is what this kernel's time used
+// to be; with kShared the three arrays live in shared memory (12 bytes per variate) and global memory only sees
+// coalesced reads and writes.  Rows too long for that work on the global arrays directly.
+template <bool kShared>
+__global__ void __launch_bounds__(kTailThreads) select_group_kernel(const SelectParams P) {
+    extern __shared__ int32_t s_rows[];
     chain_wait();
     chain_release();
     const int s = blockIdx.x, N = P.N;
     const int32_t* lt = P.lt + static_cast<size_t>(s) * N;
-    const int32_t* eq = P.eq + static_cast<size_t>(s) * N;
+    int32_t* eq = P.eq + static_cast<size_t>(s) * N;
     int32_t* members = P.members + static_cast<size_t>(s) * N;
     int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
     int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
     uint32_t* prio = P.prio + static_cast<size_t>(s) * N;
-    // every loop of this tail takes eight positions per thread at a time: the loads of a batch are issued together, so a
-    // batch costs one or two memory round trips instead of one per position
-    for (int base = 0; base < N; base += 8 * kSelThreads) {
-        int dst[8];
+    int32_t* gid_by_pos = P.lt + static_cast<size_t>(s) * N;       // lt is dead after the first pass: group id by position
+    int32_t* w_eq = kShared ? s_rows : eq;                         // working copies, by variate / position / variate
+    int32_t* w_members = kShared ? s_rows + N : members;
+    int32_t* w_gid = kShared ? s_rows + 2 * N : gid;
+    // every loop of this kernel takes several positions per thread at a time: the loads of a batch are issued together, so
+    // a batch costs one or two memory round trips instead of one per position
+    constexpr int U = 4;
+    for (int base = 0; base < N; base += U * kTailThreads) {
+        int dst[U], rank[U];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = base + u * kSelThreads + static_cast<int>(threadIdx.x);
-            dst[u] = i < N ? __ldcg(lt + i) + __ldcg(eq + i) : -1;
+        for (int u = 0; u < U; ++u) {
+            const int i = base + u * kTailThreads + static_cast<int>(threadIdx.x);
+            rank[u] = i < N ? __ldcg(eq + i) : 0;
+            dst[u] = i < N ? __ldcg(lt + i) + rank[u] : -1;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (dst[u] >= 0) members[dst[u]] = base + u * kSelThreads + static_cast<int>(threadIdx.x);
+        for (int u = 0; u < U; ++u) {
+            const int i = base + u * kTailThreads + static_cast<int>(threadIdx.x);
+            if (dst[u] >= 0) {
+                w_members[dst[u]] = i;
+                if (kShared) w_eq[i] = rank[u];
+            }
+        }
     }
     __syncthreads();
     // group heads over the sorted positions: the first member of every group has no equal key before it
-    const int total_groups = ordered_compact(
-        N, [&](int p, int* nn) { *nn = __ldcg(members + p); return __ldcg(eq + *nn) == 0; },
+    const int total_groups = ordered_compact<kTailThreads, kTailChunks>(
+        N, [&](int p, int* nn) { *nn = w_members[p]; return w_eq[*nn] == 0; },
         [&](int p, bool head, int before, int nn) {
             if (head) off[before] = p;
-            gid[nn] = before - (head ? 0 : 1);           // heads at or below p, minus one
+            const int g = before - (head ? 0 : 1);       // heads at or below p, minus one
+            w_gid[nn] = g;
+            gid_by_pos[p] = g;
+            if (kShared) members[p] = nn;
         });
     for (int i = total_groups + threadIdx.x; i <= N; i += blockDim.x) off[i] = N;
     if (threadIdx.x == 0) P.n_groups[s] = total_groups;
     __syncthreads();
-    for (int base = 0; base < N; base += 8 * kSelThreads) {
-        int nn[8], rank[8], g[8];
+    for (int base = 0; base < N; base += U * kTailThreads) {
+        int rank[U], g[U];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int p = base + u * kSelThreads + static_cast<int>(threadIdx.x);
-            nn[u] = p < N ? __ldcg(members + p) : 0;
+        for (int u = 0; u < U; ++u) {
+            const int p = base + u * kTailThreads + static_cast<int>(threadIdx.x);
+            const int nn = p < N ? w_members[p] : 0;
+            rank[u] = w_eq[nn];
+            g[u] = w_gid[nn];
+            if (kShared && p < N) gid[p] = w_gid[p];     // position p doubles as a variate index for the copy-out
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            rank[u] = __ldcg(eq + nn[u]);
-            g[u] = __ldcg(gid + nn[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int p = base + u * kSelThreads + static_cast<int>(threadIdx.x);
+        for (int u = 0; u < U; ++u) {
+            const int p = base + u * kTailThreads + static_cast<int>(threadIdx.x);
             if (p < N)
                 prio[p] = philox4x32_10_word0(static_cast<uint32_t>(rank[u]), static_cast<uint32_t>(g[u]), static_cast<uint32_t>(s), P.step,
                                               P.seed_lo, P.seed_hi);
@@ -231,20 +269,20 @@ __global__ void __launch_bounds__(kSelThreads) select_group_kernel(const SelectP
     }
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const SelectParams P) {
+__global__ void __launch_bounds__(kTailThreads) select_sample_kernel(const SelectParams P) {
     __shared__ int flag;
     chain_wait();
     chain_release();
     const int s = blockIdx.z, N = P.N;
     const int32_t* members = P.members + static_cast<size_t>(s) * N;
-    const int32_t* gid = P.group_id + static_cast<size_t>(s) * N;
+    const int32_t* gid_by_pos = P.lt + static_cast<size_t>(s) * N;      // written by select_group_kernel
     const int32_t* off = P.group_offsets + static_cast<size_t>(s) * (N + 1);
     const uint32_t* prio = P.prio + static_cast<size_t>(s) * N;
     int32_t* keep = P.keep + static_cast<size_t>(s) * N;
-    const int p = blockIdx.x * kSelThreads + threadIdx.x;
+    const int p = blockIdx.x * kTailThreads + threadIdx.x;
     if (p < N) {
         const int nn = members[p];
-        const int g = gid[nn];
+        const int g = gid_by_pos[p];
         const int begin = off[g], end = off[g + 1];
         const uint32_t mine = prio[p];
         int smaller = 0;
@@ -259,7 +297,7 @@ __global__ void __launch_bounds__(kSelThreads) select_sample_kernel(const Select
     // ---- the last CTA of this hash row: compaction of the kept variates in ascending index order --------
     int32_t* sel = P.sel_idx + static_cast<size_t>(s) * N;
     int32_t* inv = P.inv_idx + static_cast<size_t>(s) * N;
-    const int total = ordered_compact(
+    const int total = ordered_compact<kTailThreads, kTailChunks>(
         N, [&](int i, int*) { return __ldcg(keep + i) != 0; },
         [&](int i, bool kept, int before, int) {
             if (kept) sel[before] = i;
@@ -511,15 +549,30 @@ int select_launch(const uint64_t* keys, const vardrop_select_cfg& c, int32_t* gr
         { LaunchScope ls_(K_SELECT_SMALL, stream); err = launch_chained(select_small_kernel, dim3(c.S), dim3(M / 2), smem, stream, P, M); }
         return check_cuda(err, "select: launch");
     }
-    if (int st = check_cuda(cudaMemsetAsync(base, 0, w.zero_begin + w.zero_bytes, stream), "select: clear counters")) return st;
+    if (int st = check_cuda(cudaMemsetAsync(base + w.zero_begin, 0, w.zero_bytes, stream), "select: clear counters")) return st;
     const dim3 grid1((c.N + kSelThreads - 1) / kSelThreads, (c.N + kKeyChunk - 1) / kKeyChunk, c.S);
     cudaError_t err;
     { LaunchScope ls_(K_SELECT_COUNT, stream); err = launch_chained(select_count_kernel, grid1, dim3(kSelThreads), 0, stream, P); }
     if (int st = check_cuda(err, "select: count launch")) return st;
-    { LaunchScope ls_(K_SELECT_GROUP, stream); err = launch_chained(select_group_kernel, dim3(c.S), dim3(kSelThreads), 0, stream, P); }
+    const size_t group_smem = 3 * sizeof(int32_t) * static_cast<size_t>(c.N);
+    if (group_smem <= kGroupMaxSmem) {
+        static thread_local int group_attr_dev = -1;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (group_attr_dev != dev) {
+            if (int st = check_cuda(cudaFuncSetAttribute(select_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kGroupMaxSmem)),
+                                    "select: smem attribute")) return st;
+            group_attr_dev = dev;
+        }
+        LaunchScope ls_(K_SELECT_GROUP, stream);
+        err = launch_chained(select_group_kernel<true>, dim3(c.S), dim3(kTailThreads), group_smem, stream, P);
+    } else {
+        LaunchScope ls_(K_SELECT_GROUP, stream);
+        err = launch_chained(select_group_kernel<false>, dim3(c.S), dim3(kTailThreads), 0, stream, P);
+    }
     if (int st = check_cuda(err, "select: group launch")) return st;
-    const dim3 grid2((c.N + kSelThreads - 1) / kSelThreads, 1, c.S);
-    { LaunchScope ls_(K_SELECT_SAMPLE, stream); err = launch_chained(select_sample_kernel, grid2, dim3(kSelThreads), 0, stream, P); }
+    const dim3 grid2((c.N + kTailThreads - 1) / kTailThreads, 1, c.S);
+    { LaunchScope ls_(K_SELECT_SAMPLE, stream); err = launch_chained(select_sample_kernel, grid2, dim3(kTailThreads), 0, stream, P); }
     return check_cuda(err, "select: sample launch");
 }
 

@@ -60,6 +60,22 @@ def test_select_group_sizes_around_the_counting_limit():
             check(keys, gs, rate, seed=99, step=4)
 
 
+def test_select_long_rows():
+    """Rows beyond the one-CTA path: grouping with its working arrays in shared memory (up to 18432 variates), at that
+    limit, and on the global arrays beyond it; several rows at once; one group only and all-distinct keys."""
+    for N, G in ((18432, 700), (18433, 50), (24000, 3000)):
+        check(inputs.make_keys(N, G, k=4, f_hi=169, seed=N), 10, 1.0, seed=42, step=2)
+    rows = np.stack([inputs.make_keys(2500, 30 + 40 * s, k=3, f_hi=49, seed=90 + s) for s in range(3)])
+    check(rows, 0, 0.25, seed=7, step=1)
+    rows = np.stack([inputs.make_keys(19000, 100 + 900 * s, k=4, f_hi=169, seed=190 + s) for s in range(2)])
+    check(rows, 4, 0.5, seed=8, step=6)
+    got = check(np.full(5000, 77, dtype=np.uint64), 0, 0.1, seed=3, step=0)
+    assert got["n_groups"][0] == 1 and got["n_sel"][0] == 500
+    distinct = np.arange(1, 4097, dtype=np.uint64)[np.random.default_rng(1).permutation(4096)]
+    got = check(distinct, 10, 1.0, seed=1, step=0)
+    assert got["n_groups"][0] == 4096 and got["n_sel"][0] == 4096
+
+
 def test_select_multiple_scopes():
     rows = np.stack([inputs.make_keys(500, 20 + s, k=3, f_hi=25, seed=s) for s in range(5)])
     got = check(rows, 5, 1.0, seed=77, step=3)
