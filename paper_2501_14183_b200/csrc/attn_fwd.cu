@@ -193,6 +193,30 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Two fp32 values in one 64-bit register pair, for the packed fp32 instructions of sm_100 (one issue slot for two results;
+// each half is the IEEE operation of the scalar instruction, so results do not change).
+__device__ __forceinline__ uint64_t pair_of(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void halves_of(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma_pair(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_pair(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<const uint32_t*>(&v);
@@ -350,15 +374,29 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
 #pragma unroll
             for (int i = 0; i < 8; ++i) mx[i] = s[i];
 #pragma unroll
-            for (int i = 8; i < kTile; ++i) mx[i & 7] = fmaxf(mx[i & 7], s[i]);
-            const float m_tile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+            for (int i = 8; i < kTile - 8; i += 16) {             // three-input maximum: two new values per instruction
+#pragma unroll
+                for (int u = 0; u < 8; ++u) mx[u] = max3(mx[u], s[i + u], s[i + 8 + u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], s[kTile - 8 + u]);
+            const float m_tile = fmaxf(max3(mx[0], mx[1], mx[2]), max3(max3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
             const float m_new = fmaxf(m_run, m_tile * P.scale_log2);
             alpha = fast_exp2(m_run - m_new);
-            float l4[4] = {0.f, 0.f, 0.f, 0.f};
+            float l4[4];
+            {
+                const uint64_t scale2 = pair_of(P.scale_log2, P.scale_log2), shift2 = pair_of(-m_new, -m_new);
+                uint64_t l2[2] = {pair_of(0.f, 0.f), pair_of(0.f, 0.f)};          // four running sums: keys i = 0..3 mod 4
 #pragma unroll
-            for (int i = 0; i < kTile; ++i) {                     // exp2(-inf) = 0 for the masked keys
-                s[i] = fast_exp2(fmaf(s[i], P.scale_log2, -m_new));
-                l4[i & 3] += s[i];
+                for (int i = 0; i < kTile; i += 2) {              // exp2(-inf) = 0 for the masked keys
+                    float x0, x1;
+                    halves_of(fma_pair(pair_of(s[i], s[i + 1]), scale2, shift2), x0, x1);
+                    s[i] = fast_exp2(x0);
+                    s[i + 1] = fast_exp2(x1);
+                    l2[(i >> 1) & 1] = add_pair(l2[(i >> 1) & 1], pair_of(s[i], s[i + 1]));
+                }
+                halves_of(l2[0], l4[0], l4[1]);
+                halves_of(l2[1], l4[2], l4[3]);
             }
 #pragma unroll
             for (int c = 0; c < 4; ++c) store_row_chunk32(sP, tid, c * 32, s + c * 32);
@@ -391,7 +429,8 @@ __global__ void __launch_bounds__(kFwdThreads) attn_fwd_kernel(const __grid_cons
                 for (int c = 0; c < kDP / 32; ++c) tmem_ld32(tmem_o + lane_sel + c * 32, ov + c * 32);
                 tmem_ld_wait();
 #pragma unroll
-                for (int d = 0; d < kDP; ++d) o_acc[d] = fmaf(o_acc[d], alpha, ov[d]);     // rescale and add in one step
+                for (int d = 0; d < kDP; d += 2)                                          // rescale and add in one step
+                    halves_of(fma_pair(pair_of(o_acc[d], o_acc[d + 1]), pair_of(alpha, alpha), pair_of(ov[d], ov[d + 1])), o_acc[d], o_acc[d + 1]);
             }
             tc_fence_before();
             ok = __syncthreads_and(ok);                  // a wait gave up somewhere in the CTA: stop issuing work
