@@ -403,7 +403,22 @@ __global__ void __launch_bounds__(kSmallMaxN / 2) select_small_kernel(const Sele
 
     uint64_t k0 = p0 < N ? keys[p0] : ~0ull, k1 = p1 < N ? keys[p1] : ~0ull;
     uint32_t n0 = p0, n1 = p1;
-    bitonic_sort_regs<true>(k0, n0, k1, n1, a, idx, M);
+    // Keys of up to 53 bits (k <= 4 frequencies of 12 bits, say) leave room for the variate index below them: one 64-bit
+    // word per item orders by (key, index), and the sort moves a third less data per compare-exchange.
+    constexpr int kIndexBits = 11;
+    static_assert((1 << kIndexBits) >= kSmallMaxN, "index field too narrow");
+    const bool wide = __syncthreads_or((p0 < N && (k0 >> (64 - kIndexBits)) != 0) || (p1 < N && (k1 >> (64 - kIndexBits)) != 0));
+    if (!wide) {
+        if (p0 < N) k0 = (k0 << kIndexBits) | n0;
+        if (p1 < N) k1 = (k1 << kIndexBits) | n1;
+        bitonic_sort_regs<false>(k0, n0, k1, n1, a, idx, M);
+        n0 = static_cast<uint32_t>(k0) & ((1u << kIndexBits) - 1u);       // padding items (all ones) sort last and are never read
+        n1 = static_cast<uint32_t>(k1) & ((1u << kIndexBits) - 1u);
+        k0 >>= kIndexBits;
+        k1 >>= kIndexBits;
+    } else {
+        bitonic_sort_regs<true>(k0, n0, k1, n1, a, idx, M);
+    }
     a[p0] = k0; a[p1] = k1; idx[p0] = n0; idx[p1] = n1;
     __syncthreads();
 
