@@ -80,6 +80,14 @@ def test_attention_all_tokens(B, N, H, D):
     check_case(B, N, H, D, None, 1.0, seed=N)
 
 
+@pytest.mark.parametrize("B,N,H,D,Ns", [(1, 512, 2, 64, 200), (1, 513, 2, 64, 200), (1, 512, 2, 64, 256), (1, 512, 1, 64, 384),
+                                        (1, 512, 1, 64, 512), (1, 640, 2, 32, 384), (2, 1100, 1, 64, 640)])
+def test_attention_selected_at_path_boundaries(B, N, H, D, Ns):
+    """Both sides of the largest N whose kept rows are gathered by the tile loads themselves (512), kept counts that fill
+    whole tiles exactly (two, three, four tiles on the gathered path; three and five on the staged one), head size 32."""
+    check_case(B, N, H, D, pick(N, Ns, seed=N * 3 + Ns), 1.0, seed=N + 11 * Ns)
+
+
 def test_attention_identity_selection_equals_all_token_path():
     B, N, H, D = 1, 200, 2, 64
     dev, _ = bf16_tokens(B, N, H, D, 1.0, seed=3)
