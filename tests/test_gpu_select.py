@@ -76,6 +76,21 @@ def test_select_long_rows():
     assert got["n_groups"][0] == 4096 and got["n_sel"][0] == 4096
 
 
+def test_select_random_configurations():
+    """Seeded random draws of (N, rows, groups, gs, rate, k) on both sides of every size limit of the kernels
+    (2048: one-CTA path; 18432: grouping in shared memory; 65536: the largest N)."""
+    rng = np.random.default_rng(123)
+    for it in range(24):
+        N = int(rng.choice([63, 64, 65, 700, 2047, 2048, 2049, 4096, 8192, 18432, 18433, 30000, 65536]))
+        S = int(rng.choice([1, 1, 2, 3])) if N <= 20000 else 1
+        G = int(rng.integers(1, max(2, N // int(rng.choice([1, 2, 8, 50, 400])))))
+        gs = int(rng.choice([0, 1, 3, 10, 100]))
+        rate = float(rng.choice([0.05, 0.2, 0.5, 1.0]))
+        k = int(rng.choice([3, 4, 5]))
+        rows = np.stack([inputs.make_keys(N, G, k=k, f_hi=int(rng.choice([25, 49, 169, 361])), seed=1000 * it + s) for s in range(S)])
+        check(rows, gs, rate, seed=int(rng.integers(0, 2**62)), step=int(rng.integers(0, 1000)))
+
+
 def test_select_multiple_scopes():
     rows = np.stack([inputs.make_keys(500, 20 + s, k=3, f_hi=25, seed=s) for s in range(5)])
     got = check(rows, 5, 1.0, seed=77, step=3)
