@@ -88,6 +88,37 @@ def test_attention_selected_at_path_boundaries(B, N, H, D, Ns):
     check_case(B, N, H, D, pick(N, Ns, seed=N * 3 + Ns), 1.0, seed=N + 11 * Ns)
 
 
+def test_attention_random_configurations():
+    """Seeded random draws of (B, N, H, D, kept count, value scale): gathered, staged and all-token paths, one to six tiles.
+    Value scales stay at or below 1: the absolute tolerance is stated for unit-scale tokens (bf16 rounding of P and dS is
+    relative, so gradients of larger tokens carry proportionally larger absolute errors)."""
+    rng = np.random.default_rng(2025)
+    for it in range(14):
+        N = int(rng.integers(2, 760))
+        D = int(rng.choice([64, 64, 32]))
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        Ns = int(rng.integers(1, N + 1))
+        sel = None if it % 4 == 3 else pick(N, Ns, seed=it)
+        check_case(B, N, H, D, sel, float(rng.choice([1.0, 0.3536, 0.6])), seed=500 + it)
+
+
+@pytest.mark.parametrize("B,N,H,D,Ns,std", [(3, 341, 2, 32, 326, 2.0), (2, 604, 1, 64, 210, 2.0), (1, 300, 2, 64, None, 3.0)])
+def test_attention_large_tokens_relative_error(B, N, H, D, Ns, std):
+    """Tokens a few times the unit scale: peaky softmax rows and gradients of tens.  The errors of the bf16 products are
+    relative, so the bound is the unit-scale tolerance times the largest magnitude of the tensor."""
+    dev, ref = bf16_tokens(B, N, H, D, std, seed=N + 5)
+    sel = None if Ns is None else pick(N, Ns, seed=N)
+    o, lse, dq, dk, dv, status, _ = run_attention(dev, B, N, H, D, sel)
+    assert status == vd.OK
+    n_rows = N if sel is None else len(sel)
+    wo, wl = oracle.attn_fwd(ref[0], ref[1], ref[2], sel)
+    wq, wk, wv = oracle.attn_bwd(ref[0], ref[1], ref[2], ref[3][:, :n_rows], sel)
+    for got, want, name in ((o, wo, "o"), (lse, wl, "lse"), (dq, wq, "dq"), (dk, wk, "dk"), (dv, wv, "dv")):
+        bound = 2e-2 * max(1.0, float(np.abs(want).max()))
+        err = float(np.abs(got - want).max())
+        assert np.all(np.isfinite(got)) and err <= bound, f"{name}: max abs error {err:.3e} > {bound:.3e}"
+
+
 def test_attention_identity_selection_equals_all_token_path():
     B, N, H, D = 1, 200, 2, 64
     dev, _ = bf16_tokens(B, N, H, D, 1.0, seed=3)
