@@ -64,6 +64,39 @@ def test_hash_parity_small(B, N, L, k, scope):
     np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
 
 
+def _largest_prime_factor(n):
+    p, best = 2, 1
+    while n > 1:
+        if n % p == 0:
+            best, n = p, n // p
+        else:
+            p += 1
+    return best
+
+
+def test_hash_random_configurations():
+    """Seeded random draws of (B, N, L, k, scope): the register-blocked transforms (L = 96, 192, 336, 720) with every team
+    size, and the generic kernel at window lengths with any mix of the supported factors 2, 3, 5, 7 (odd lengths and powers
+    of two included; a length with a larger prime factor is refused, see test_hash_argument_errors)."""
+    smooth = [n for n in range(12, 900) if _largest_prime_factor(n) <= 7]
+    rng = np.random.default_rng(77)
+    for it in range(20):
+        L = int(rng.choice([96, 192, 336, 720])) if it % 2 == 0 else int(rng.choice(smooth))
+        B, N = int(rng.integers(1, 40)), int(rng.integers(1, 260))
+        k = int(rng.integers(1, 6))
+        scope = int(rng.integers(0, 2))
+        nb = L // 2 + 1
+        f_lo, f_hi = (0, nb) if (nb + 1) // 2 - 1 < k + 1 else (0, 0)
+        if nb - 1 < k + 1:
+            continue
+        x = random_periodic(B, N, L, k, seed=9000 + it)
+        x, keys, freqs, abar, _ = gap_filtered_windows(x, k, f_lo, f_hi, scope)
+        gk, gf, ga = run_hash(x, k, f_lo, f_hi, scope)
+        assert np.array_equal(gf, freqs), (B, N, L, k, scope)
+        assert np.array_equal(gk, keys), (B, N, L, k, scope)
+        np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
+
+
 @pytest.mark.parametrize("name", ["tiny", "elec", "traffic", "long", "scale"])
 def test_hash_parity_workloads(name):
     w = inputs.WORKLOADS[name]
