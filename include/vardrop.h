@@ -41,7 +41,7 @@ extern "C" {
 typedef enum {
     VARDROP_OK = 0,
     VARDROP_ERR_INVALID_ARG = 1,   /* null/misaligned pointer, size out of range                       */
-    VARDROP_ERR_UNSUPPORTED = 2,   /* e.g. L with a prime factor above 7, head dimension other than 32/64 */
+    VARDROP_ERR_UNSUPPORTED = 2,   /* e.g. L above 8192, head dimension other than 32/64 */
     VARDROP_ERR_WORKSPACE = 3,     /* ws_bytes below the *_workspace_bytes answer                      */
     VARDROP_ERR_CUDA = 4,          /* a CUDA runtime call or launch failed                             */
     VARDROP_ERR_TIMEOUT = 5,       /* device side: a bounded wait gave up (device status word only)    */
@@ -86,7 +86,8 @@ int vardrop_profile_read(int id, double* total_ms, long long* launches);
  *
  * cfg (host)  B, N, L  shape of x;  1 <= k <= 5;  f_lo/f_hi candidate band, both 0 selects the default
  *             f_lo = 1, f_hi = ceil((L/2+1)/2) (25 at L = 96, the cut-off of Appendix E);
- *             requires 0 <= f_lo, f_lo + k <= f_hi <= L/2+1, f_hi <= 4096, L <= 8192 and L a product of 2, 3, 5, 7.
+ *             requires 0 <= f_lo, f_lo + k <= f_hi <= L/2+1, f_hi <= 4096 and L <= 8192 (prime factors of L above 7 are
+ *             transformed as plain sums, at a cost that grows with the factor).
  * x           [B, N, L] float32, contiguous.
  * keys        [S, N] uint64 out.
  * freqs       [S, N, k] int32 out, the ranked bins; may be NULL.

@@ -5,7 +5,7 @@
 // per-instance scope) and all the windows that feed them, so the mean over the batch never leaves the SM
 // and is summed in ascending instance order.  Two real windows ride one complex transform
 // (z = x1 + i x2; X1_f = (Z_f + conj Z_{L-f}) / 2, X2_f = (Z_f - conj Z_{L-f}) / 2i), which is evaluated by
-// a Stockham autosort mixed-radix FFT (radices 4, 2, 3, 5, 7) whose butterflies are spread over the
+// a Stockham autosort mixed-radix FFT (radices 4, 2, 3, 5, 7; larger prime factors as plain sums) whose butterflies are spread over the
 // whole CTA.  Twiddles are produced once per CTA in double precision.
 #include "common.cuh"
 #include "kernels.h"
@@ -43,6 +43,8 @@ __device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(
 template <int R>
 __device__ __forceinline__ void small_dft(float2* v);
 
+template <>
+__device__ __forceinline__ void small_dft<1>(float2*) {}      // the copy-in stage of a length without small factors
 template <>
 __device__ __forceinline__ void small_dft<2>(float2* v) {
     const float2 a = v[0], b = v[1];
@@ -142,6 +144,35 @@ __device__ __forceinline__ void fft_stage(const float2* __restrict__ in, float2*
     }
 }
 
+// The same stage for any radix R (a prime factor above 7), as the plain sum it stands for: one thread per output point
+// adds its R inputs times table twiddles.  Output m of butterfly j needs w^(r (kk L/(Ns R) + m L/R)) for input r: the
+// exponent advances by a fixed step per input, taken modulo L by one conditional subtraction.  O(L R) per transform.
+__device__ __forceinline__ void fft_stage_any(const float2* __restrict__ in, float2* __restrict__ out, const float2* __restrict__ tw,
+                                              int n_fft, int L, int R, FastDiv div_lr, FastDiv div_ns) {
+    const uint32_t LR = div_lr.d, Ns = div_ns.d, uL = static_cast<uint32_t>(L), uR = static_cast<uint32_t>(R);
+    const uint32_t tw_step = uL / (Ns * uR), m_step = uL / uR;
+    const uint32_t total = static_cast<uint32_t>(n_fft) * uL;
+    for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+        const uint32_t bj = t / uR, m = t - bj * uR;           // m fastest: the threads of a butterfly share its inputs
+        const uint32_t p = fd_div(bj, div_lr);
+        const uint32_t j = bj - p * LR;
+        const uint32_t q = fd_div(j, div_ns);
+        const uint32_t kk = j - q * Ns;
+        const uint32_t step = (kk * tw_step + m * m_step) % uL;
+        const float2* src = in + p * uL + j;
+        float2 acc = src[0];
+        uint32_t e = 0;
+        for (uint32_t r = 1; r < uR; ++r) {
+            e += step;
+            if (e >= uL) e -= uL;
+            const float2 v = src[r * LR], w = tw[e];
+            acc.x = fmaf(v.x, w.x, fmaf(-v.y, w.y, acc.x));
+            acc.y = fmaf(v.x, w.y, fmaf(v.y, w.x, acc.y));
+        }
+        out[p * uL + q * Ns * uR + kk + m * Ns] = acc;
+    }
+}
+
 // First Stockham stage (Ns = 1: no twiddles, butterfly j writes out[j R + r]) reading the windows straight from global
 // memory: transform p carries window 2p of the pass in its real part and window 2p + 1 (if any) in its imaginary part.
 template <int R>
@@ -207,7 +238,8 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
             case 3: fft_first_stage<3>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
             case 4: fft_first_stage<4>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
             case 5: fft_first_stage<5>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
-            default: fft_first_stage<7>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            case 7: fft_first_stage<7>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;
+            default: fft_first_stage<1>(P, cur, n_win, row0, b0, cw, P.div_lr[0]); break;      // plain copy-in: every factor is a large prime
         }
         __syncthreads();
         for (int s = 1; s < P.n_stages; ++s) {
@@ -216,7 +248,8 @@ __global__ void __launch_bounds__(kHashThreads) hash_kernel(const HashParams P) 
                 case 3: fft_stage<3>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
                 case 4: fft_stage<4>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
                 case 5: fft_stage<5>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
-                default: fft_stage<7>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
+                case 7: fft_stage<7>(cur, oth, tw, n_fft, L, P.div_lr[s], P.div_ns[s]); break;
+                default: fft_stage_any(cur, oth, tw, n_fft, L, P.radix[s], P.div_lr[s], P.div_ns[s]); break;
             }
             __syncthreads();
             float2* tmp = cur; cur = oth; oth = tmp;
@@ -299,9 +332,6 @@ int hash_validate(const vardrop_hash_cfg& c, int* f_lo, int* f_hi) {
     if (lo == 0 && hi == 0) { lo = 1; hi = (nb + 1) / 2; }
     if (lo < 0 || hi > nb || hi > 4096 || lo + c.k > hi)
         return fail(VARDROP_ERR_INVALID_ARG, "hash: band [%d,%d) needs 0 <= f_lo, f_lo + k <= f_hi <= min(L/2+1, 4096)", lo, hi);
-    int rem = c.L;
-    for (int p : {2, 3, 5, 7}) while (rem % p == 0) rem /= p;
-    if (rem != 1) return fail(VARDROP_ERR_UNSUPPORTED, "hash: L=%d has a prime factor above 7", c.L);
     if (static_cast<long long>(c.B) * c.N > (1ll << 31) - 1) return fail(VARDROP_ERR_INVALID_ARG, "hash: B*N too large");
     *f_lo = lo; *f_hi = hi;
     return VARDROP_OK;
@@ -321,7 +351,8 @@ int hash_launch(const float* x, const vardrop_hash_cfg& c, uint64_t* keys, int32
     P.rows_total = c.scope == 0 ? c.N : c.B * c.N;
     P.win_per_row = c.scope == 0 ? c.B : 1;
 
-    // radix plan: fours first, then a two, then the odd primes
+    // radix plan: fours first, then a two, then the odd primes; prime factors above 7 come last as plain-sum stages (behind
+    // a copy-in stage when there is no small factor to read the windows with)
     int rem = c.L, ns = 1;
     P.n_stages = 0;
     auto push = [&](int r) {
@@ -333,6 +364,8 @@ int hash_launch(const float* x, const vardrop_hash_cfg& c, uint64_t* keys, int32
     };
     while (rem % 4 == 0) { push(4); rem /= 4; }
     for (int p : {2, 3, 5, 7}) while (rem % p == 0) { push(p); rem /= p; }
+    if (rem > 1 && P.n_stages == 0) push(1);
+    for (int p = 11; rem > 1; p += 2) while (rem % p == 0) { push(p); rem /= p; }
 
     // windows per pass: about 2048 complex points per buffer, an even count
     int per_pass = 2 * (2048 / c.L);

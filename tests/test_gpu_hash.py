@@ -46,6 +46,8 @@ SHAPES = [
     (7, 19, 720, 5, 0), (2, 13, 48, 2, 0), (3, 11, 30, 2, 0), (2, 5, 14, 1, 0), (4, 8, 64, 3, 0), (3, 6, 2048, 5, 0),
     (70, 3, 96, 3, 0), (4, 21, 96, 2, 1), (3, 10, 336, 4, 1), (5, 7, 720, 5, 1), (1, 300, 96, 3, 0), (2, 4, 210, 3, 0),
     (6, 17, 192, 3, 0), (9, 40, 192, 4, 0), (17, 23, 336, 4, 0), (2, 1300, 96, 3, 0), (33, 300, 96, 3, 0),
+    # window lengths with prime factors above 7 (plain-sum stages): 2 * 47, 4 * 3 * 19, a prime, 11 * 13, 2 * 1021
+    (3, 10, 94, 3, 0), (2, 7, 228, 3, 0), (2, 5, 733, 4, 0), (3, 6, 143, 2, 1), (1, 3, 2042, 5, 0),
 ]
 
 
@@ -64,24 +66,12 @@ def test_hash_parity_small(B, N, L, k, scope):
     np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
 
 
-def _largest_prime_factor(n):
-    p, best = 2, 1
-    while n > 1:
-        if n % p == 0:
-            best, n = p, n // p
-        else:
-            p += 1
-    return best
-
-
 def test_hash_random_configurations():
     """Seeded random draws of (B, N, L, k, scope): the register-blocked transforms (L = 96, 192, 336, 720) with every team
-    size, and the generic kernel at window lengths with any mix of the supported factors 2, 3, 5, 7 (odd lengths and powers
-    of two included; a length with a larger prime factor is refused, see test_hash_argument_errors)."""
-    smooth = [n for n in range(12, 900) if _largest_prime_factor(n) <= 7]
+    size, and the generic kernel at window lengths of any factorisation (odd, prime, powers of two)."""
     rng = np.random.default_rng(77)
     for it in range(20):
-        L = int(rng.choice([96, 192, 336, 720])) if it % 2 == 0 else int(rng.choice(smooth))
+        L = int(rng.choice([96, 192, 336, 720])) if it % 2 == 0 else int(rng.integers(12, 900))
         B, N = int(rng.integers(1, 40)), int(rng.integers(1, 260))
         k = int(rng.integers(1, 6))
         scope = int(rng.integers(0, 2))
@@ -155,7 +145,7 @@ def test_hash_argument_errors():
     ws = vd.alloc_ws(256)
     keys = torch.empty((1, 4), dtype=torch.int64, device="cuda")
     for cfg, status in [(vd.HashCfg(2, 4, 96, 0, 0, 0, 0), vd.ERR_INVALID_ARG), (vd.HashCfg(2, 4, 96, 6, 0, 0, 0), vd.ERR_INVALID_ARG),
-                        (vd.HashCfg(2, 4, 94, 3, 0, 0, 0), vd.ERR_UNSUPPORTED),      # 94 = 2 * 47
+                        (vd.HashCfg(2, 4, 8200, 3, 0, 0, 0), vd.ERR_UNSUPPORTED),    # windows above 8192 points
                         (vd.HashCfg(2, 4, 96, 3, 10, 12, 0), vd.ERR_INVALID_ARG), (vd.HashCfg(2, 4, 96, 3, 0, 60, 0), vd.ERR_INVALID_ARG),
                         (vd.HashCfg(2, 4, 96, 3, 0, 0, 2), vd.ERR_INVALID_ARG)]:
         with pytest.raises(vd.VardropError) as e:

@@ -64,8 +64,8 @@ def test_workspace_queries_need_no_gpu(lib):
 
 def test_host_side_validation_needs_no_gpu(lib):
     # argument checks run before any CUDA call: bad configs are rejected on a machine without a GPU too
-    st = lib.vardrop_hash(None, C.byref(vd.HashCfg(2, 4, 94, 3, 0, 0, 0)), None, None, None, None, 0, None)
-    assert st == vd.ERR_UNSUPPORTED and b"prime factor" in lib.vardrop_last_error()
+    st = lib.vardrop_hash(None, C.byref(vd.HashCfg(2, 4, 8200, 3, 0, 0, 0)), None, None, None, None, 0, None)
+    assert st == vd.ERR_UNSUPPORTED and b"above 8192" in lib.vardrop_last_error()
     st = lib.vardrop_hash(None, C.byref(vd.HashCfg(2, 4, 96, 3, 0, 0, 0)), None, None, None, None, 0, None)
     assert st == vd.ERR_INVALID_ARG and b"x is NULL" in lib.vardrop_last_error()
     st = lib.vardrop_attn_fwd(None, None, None, None, None, C.byref(vd.AttnCfg(1, 8, 1, 48, 0.0)), None, None, None, 0, None)
