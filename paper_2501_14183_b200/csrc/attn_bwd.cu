@@ -141,6 +141,25 @@ __device__ __forceinline__ bool group3_sync_and(bool ok) {
     return r != 0;
 }
 
+// Two fp32 values in one 64-bit register pair, for the packed fp32 instructions of sm_100 (one issue slot for two results;
+// each half is the IEEE operation of the scalar instruction, so results do not change).
+__device__ __forceinline__ uint64_t pair_of(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void halves_of(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma_pair(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul_pair(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -179,7 +198,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     uint64_t* bar_ds = bars + 9;                    // dS^T of a query tile written by every worker thread
     uint64_t* bar_conv = bars + 10;                 // the "last key tile of its (instance, head)" flag of an item is written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 96);
-    float* s_stat = reinterpret_cast<float*>(smem_dyn + 128);     // [3 stages][128] lse of the query tile, log2 domain
+    float* s_stat = reinterpret_cast<float*>(smem_dyn + 128);     // [3 stages][128] minus the lse of the query tile, log2 domain
     float* s_dpart = s_stat + kQStages * kTile;                   // [2][128] Delta of the query tile: with precomputed Delta, one array per
                                                                   // tile parity (written a barrier ahead of its use); otherwise the two
                                                                   // halves' partial sums over 32 head dimensions of dO O
@@ -326,10 +345,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         tc_commit(bar_g);
     };
 
-    // lse of query `qrow` in the log2 domain (fetched by the threads of half 0; +inf switches a missing query off)
+    // minus the lse of query `qrow` in the log2 domain (fetched by the threads of half 0; -inf switches a missing query off)
     auto load_lse = [&](int b, int h, int qrow) -> float {
         if (half != 0) return 0.f;
-        return qrow < n_sel ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * 1.4426950408889634f : INFINITY;
+        return qrow < n_sel ? P.lse[(static_cast<size_t>(b) * P.H + h) * P.N + qrow] * -1.4426950408889634f : -INFINITY;
     };
     // this thread's 32 head dimensions (64 bytes) of forward-output row `qrow`, zeros when there is no such row
     auto load_o = [&](int b, int h, int qrow, uint4* dst) {
@@ -516,6 +535,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             float pv[64];
             {   // 16 queries at a time; the next piece is read from tensor memory while the current one is processed
                 const float* lse2 = s_stat + st * kTile + half * 64;
+                const uint64_t scale2 = pair_of(P.scale_log2, P.scale_log2);
                 float sv[2][16];
                 tmem_ld16(tm_st + lane_sel + half * 64, sv[0]);
 #pragma unroll
@@ -524,11 +544,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (c < 3) tmem_ld16(tm_st + lane_sel + half * 64 + (c + 1) * 16, sv[(c + 1) & 1]);
 #pragma unroll
                     for (int x = 0; x < 16; x += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 16 + x);
-                        pv[c * 16 + x + 0] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 0], P.scale_log2, -l4.x)) : 0.f;    // rows past n_sel hold zero
-                        pv[c * 16 + x + 1] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 1], P.scale_log2, -l4.y)) : 0.f;    // keys: they must not count
-                        pv[c * 16 + x + 2] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 2], P.scale_log2, -l4.z)) : 0.f;
-                        pv[c * 16 + x + 3] = key_valid ? fast_exp2(fmaf(sv[c & 1][x + 3], P.scale_log2, -l4.w)) : 0.f;
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + c * 16 + x);       // minus lse
+                        float e0, e1, e2, e3;
+                        halves_of(fma_pair(pair_of(sv[c & 1][x + 0], sv[c & 1][x + 1]), scale2, pair_of(l4.x, l4.y)), e0, e1);
+                        halves_of(fma_pair(pair_of(sv[c & 1][x + 2], sv[c & 1][x + 3]), scale2, pair_of(l4.z, l4.w)), e2, e3);
+                        pv[c * 16 + x + 0] = key_valid ? fast_exp2(e0) : 0.f;    // rows past n_sel hold zero
+                        pv[c * 16 + x + 1] = key_valid ? fast_exp2(e1) : 0.f;    // keys: they must not count
+                        pv[c * 16 + x + 2] = key_valid ? fast_exp2(e2) : 0.f;
+                        pv[c * 16 + x + 3] = key_valid ? fast_exp2(e3) : 0.f;
                     }
                     store_chunk16(sPt, row, half * 64 + c * 16, pv + c * 16);
                 }
@@ -554,10 +577,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 #pragma unroll
                         for (int x = 0; x < 16; x += 4) {
                             const float4 da = *reinterpret_cast<const float4*>(dlt + c * 16 + x);
-                            d[x + 0] = pv[c * 16 + x + 0] * (d[x + 0] - da.x);
-                            d[x + 1] = pv[c * 16 + x + 1] * (d[x + 1] - da.y);
-                            d[x + 2] = pv[c * 16 + x + 2] * (d[x + 2] - da.z);
-                            d[x + 3] = pv[c * 16 + x + 3] * (d[x + 3] - da.w);
+                            const uint64_t minus1 = pair_of(-1.f, -1.f);               // d - Delta as fma(Delta, -1, d): one rounding, as the subtraction
+                            halves_of(mul_pair(pair_of(pv[c * 16 + x + 0], pv[c * 16 + x + 1]),
+                                               fma_pair(pair_of(da.x, da.y), minus1, pair_of(d[x + 0], d[x + 1]))), d[x + 0], d[x + 1]);
+                            halves_of(mul_pair(pair_of(pv[c * 16 + x + 2], pv[c * 16 + x + 3]),
+                                               fma_pair(pair_of(da.z, da.w), minus1, pair_of(d[x + 2], d[x + 3]))), d[x + 2], d[x + 3]);
                         }
                     } else {                             // two partial sums, one per 32 head dimensions
 #pragma unroll
