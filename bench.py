@@ -4,13 +4,14 @@
 One *step* = one pass of the whole path over one synthetic batch: vardrop_hash -> vardrop_select ->
 vardrop_attn_fwd (gather + attention) -> vardrop_attn_bwd (+ scatter), all through the C ABI.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload elec|traffic|long|scale|tiny]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload scale|traffic|long|elec|tiny]   (default: scale)
   python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...     (N > 1: one rank per GPU)
   python bench.py --impl reference ...     (the CPU oracle, as it stands, on the host cores)
 
 Rank 0 prints ONE JSON line.  `value` is variate tokens per second (B * N per step) of the whole job with inputs
 resident in HBM; `e2e` is the same with host buffers and the copies inside the timed region; `roofline` describes
-the kernel with the largest share of the step; `cpu_baseline` is the oracle timed on this machine's cores.
+the kernel with the largest share of the step; `targets` holds the all-token N = 862 attention and the k-DFH / selection /
+gather fractions from a short Traffic-shaped pass; `cpu_baseline` is the oracle timed on this machine's cores.
 """
 from __future__ import annotations
 
@@ -104,7 +105,7 @@ class Path:
     """Device buffers and the four C-ABI calls of one step; `slots` rotating input/output sets keep the working set
     larger than L2 so that every step reads its inputs from HBM."""
 
-    def __init__(self, w, device, seed, slots):
+    def __init__(self, w, device, seed, slots, host_slots=2):
         import torch
         from paper_2501_14183_b200 import binding as vd
         from paper_2501_14183_b200 import inputs
@@ -117,9 +118,11 @@ class Path:
         x = inputs.make_windows(w, seed=seed)
         toks = inputs.make_tokens(w.B, w.N, w.H, w.D, w.qkv_std, seed=seed + 1)
         for s in range(slots):
-            hx = torch.from_numpy(np.roll(x, s, axis=0).copy()).pin_memory()            # same variates, instances rotated
-            ht = [torch.from_numpy(np.roll(t, s, axis=0).copy()).to(torch.bfloat16).pin_memory() for t in toks]
-            self.host.append((hx, ht))
+            hx = torch.from_numpy(np.roll(x, s, axis=0).copy())                         # same variates, instances rotated
+            ht = [torch.from_numpy(np.roll(t, s, axis=0).copy()).to(torch.bfloat16) for t in toks]
+            if s < host_slots:                                                          # pinned copies for the end-to-end leg
+                hx, ht = hx.pin_memory(), [t.pin_memory() for t in ht]
+                self.host.append((hx, ht))
             d = dict(x=hx.to(device), q=ht[0].to(device), k=ht[1].to(device), v=ht[2].to(device), d_o=ht[3].to(device),
                      o=torch.zeros((w.B, w.N, w.H, w.D), **bf), lse=torch.zeros((w.B, w.H, w.N), dtype=torch.float32, device=device),
                      dq=torch.empty((w.B, w.N, w.H, w.D), **bf), dk=torch.empty((w.B, w.N, w.H, w.D), **bf),
@@ -130,9 +133,11 @@ class Path:
         self.hws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(self.hcfg), device)
         self.sws = vd.alloc_ws(vd.vardrop_select_workspace_bytes(self.scfg), device)
         self.aws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(self.acfg), device)
-        self.host_out = [torch.empty((w.B, w.N, w.H, w.D), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
-        self.host_sel = torch.empty((w.N + 1,), dtype=torch.int32).pin_memory()
         self.step_no = 0
+
+    def host_x(self, slot):
+        """The windows of device slot `slot` as a numpy array (slot s holds the batch rotated by s instances)."""
+        return self.dev[slot]["x"].cpu().numpy()
 
     def input_bytes(self):
         w = self.w
@@ -157,40 +162,116 @@ class Path:
         vd.vardrop_attn_bwd(d["q"], d["k"], d["v"], d["o"], d["lse"], d["d_o"], sel, nsel, inv, self.acfg, d["dq"], d["dk"], d["dv"],
                             self.aws)
 
-    def step_e2e(self, slot):
-        """Same step with host buffers: inputs copied from pinned host memory, outputs copied back."""
+    def e2e_setup(self):
+        """Streams, events and host buffers of the pipelined end-to-end step: input copies of step i + 1 and output copies of
+        step i - 1 run on their own streams beside the kernels of step i (PCIe is full duplex), two device slots and two
+        host output sets in rotation."""
+        t, w = self.torch, self.w
+        self.s_in, self.s_out = t.cuda.Stream(), t.cuda.Stream()
+        mk = lambda: [t.cuda.Event() for _ in range(2)]
+        self.ev_in, self.ev_comp, self.ev_out = mk(), mk(), mk()
+        cur = t.cuda.current_stream()
+        for e in self.ev_in + self.ev_comp + self.ev_out:
+            e.record(cur)
+        self.host_out = [[t.empty((w.B, w.N, w.H, w.D), dtype=t.bfloat16).pin_memory() for _ in range(4)] for _ in range(2)]
+        self.host_sel = [t.empty((w.N + 1,), dtype=t.int32).pin_memory() for _ in range(2)]
+
+    def e2e_begin(self):
+        t = self.torch
+        ev = t.cuda.Event()
+        ev.record()
+        self.s_in.wait_event(ev)
+        self.s_out.wait_event(ev)
+
+    def e2e_drain(self):
+        cur = self.torch.cuda.current_stream()
+        for e in self.ev_out:
+            cur.wait_event(e)
+
+    def step_e2e(self, i):
+        """Same step with host buffers: every step copies its inputs from pinned host memory and its outputs back, the
+        copies of neighbouring steps overlapping this step's kernels (one cudaMemcpyAsync per tensor)."""
+        t = self.torch
+        slot = i % 2
         d = self.dev[slot]
         hx, ht = self.host[slot]
-        d["x"].copy_(hx, non_blocking=True)
-        for name, t in zip(("q", "k", "v", "d_o"), ht):
-            d[name].copy_(t, non_blocking=True)
+        cur = t.cuda.current_stream()
+        with t.cuda.stream(self.s_in):
+            self.s_in.wait_event(self.ev_comp[slot])        # the step that last read this slot's inputs is done
+            d["x"].copy_(hx, non_blocking=True)
+            for name, src in zip(("q", "k", "v", "d_o"), ht):
+                d[name].copy_(src, non_blocking=True)
+            self.ev_in[slot].record(self.s_in)
+        cur.wait_event(self.ev_in[slot])
+        cur.wait_event(self.ev_out[slot])                   # this slot's previous outputs have left the device
         self.step(slot)
-        for h, name in zip(self.host_out, ("o", "dq", "dk", "dv")):
-            h.copy_(d[name], non_blocking=True)
-        self.host_sel[: self.w.N].copy_(self.sel["sel_idx"][0], non_blocking=True)
-        self.host_sel[self.w.N:].copy_(self.sel["n_sel"], non_blocking=True)
+        hs = self.host_sel[slot]
+        hs[: self.w.N].copy_(self.sel["sel_idx"][0], non_blocking=True)     # the selection buffers are shared by the slots:
+        hs[self.w.N:].copy_(self.sel["n_sel"], non_blocking=True)           # copied in stream order, before the next step
+        self.ev_comp[slot].record(cur)
+        with t.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_comp[slot])
+            for h, name in zip(self.host_out[slot], ("o", "dq", "dk", "dv")):
+                h.copy_(d[name], non_blocking=True)
+            self.ev_out[slot].record(self.s_out)
 
     def check_status(self):
         for ws in (self.hws, self.sws, self.aws):
-            st = self.vd.ws_status(ws)
+            st = self.vd.vardrop_ws_status(ws)
             if st != self.vd.OK:
                 raise RuntimeError(f"device status {st} after the timed region")
 
 
-def time_region(torch, fn, steps, dist_barrier):
-    """K calls of fn(i) between two CUDA events, a barrier + synchronize on both sides; milliseconds."""
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    dist_barrier()
-    torch.cuda.synchronize()
-    start.record()
-    t0 = time.perf_counter()
-    for i in range(steps):
-        fn(i)
-    time_region.host_ms = (time.perf_counter() - t0) * 1e3          # host time spent issuing the K steps
-    stop.record()
-    torch.cuda.synchronize()
-    dist_barrier()
-    return start.elapsed_time(stop)
+MIN_REGION_S = 0.3          # a timed region is repeated until it has lasted this long
+MIN_INTERVALS = 50          # and has produced at least this many event intervals
+
+
+def time_region(torch, fn, steps, dist_barrier, min_seconds=None, min_intervals=None, begin=None, drain=None):
+    """Times calls of fn(i) with CUDA events on the launching stream.
+
+    One pass is exactly `steps` calls between a barrier + synchronize on both sides, with an event after every block of
+    steps (a block is one step when steps <= 64).  Passes are repeated until the accumulated device time reaches
+    `min_seconds` and at least `min_intervals` block intervals exist.  Returns a dict: `median` and `mean` milliseconds
+    per step (median over the block intervals, mean over whole passes), `intervals`, `passes`, `total_ms`, and
+    `host_ms_per_step` (host time spent issuing the calls).  `begin()` runs right after the first event of a pass and
+    `drain()` right before its last one (used by the pipelined end-to-end step to tie its copy streams to the events)."""
+    min_seconds = MIN_REGION_S if min_seconds is None else min(min_seconds, MIN_REGION_S)
+    min_intervals = MIN_INTERVALS if min_intervals is None else min(min_intervals, MIN_INTERVALS)
+    block = max(1, steps // 64)
+    per_step, pass_ms, host_s, passes, i_global = [], [], 0.0, 0, 0
+    while True:
+        marks = [torch.cuda.Event(enable_timing=True)]
+        sizes = []
+        dist_barrier()
+        torch.cuda.synchronize()
+        marks[0].record()
+        if begin is not None:
+            begin()
+        t0 = time.perf_counter()
+        done = 0
+        while done < steps:
+            n = min(block, steps - done)
+            for _ in range(n):
+                fn(i_global)
+                i_global += 1
+            done += n
+            if drain is not None and done == steps:
+                drain()
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            marks.append(ev)
+            sizes.append(n)
+        host_s += time.perf_counter() - t0
+        torch.cuda.synchronize()
+        dist_barrier()
+        for a, b, n in zip(marks[:-1], marks[1:], sizes):
+            per_step.append(a.elapsed_time(b) / n)
+        pass_ms.append(marks[0].elapsed_time(marks[-1]))
+        passes += 1
+        if (sum(pass_ms) >= min_seconds * 1e3 and len(per_step) >= min_intervals) or passes >= 2000:
+            break
+    return {"median": float(np.median(per_step)), "mean": float(sum(pass_ms) / (passes * steps)), "intervals": len(per_step),
+            "passes": passes, "total_ms": float(sum(pass_ms)), "host_ms_per_step": host_s * 1e3 / (passes * steps)}
 
 
 def recorded_traffic(kernel, workload):
@@ -258,7 +339,6 @@ def kernel_table(per_kernel, work, peaks):
 def pearson_leg(torch, vd, path, w, peaks, barrier, args):
     """Times vardrop_pearson_max (maximum Pearson correlation per variate, Appendix A / Eq. 4) on the workload's windows and, unless
     --no-cpu, the oracle on one instance.  Algorithmic work: 2 B N^2 L flop (every pair once per direction)."""
-    import oracle
     device = path.dev[0]["x"].device
     cfg = vd.PearsonCfg(w.B, w.N, w.L, 0.9)
     out = torch.empty((w.B, w.N), dtype=torch.float32, device=device)
@@ -269,23 +349,87 @@ def pearson_leg(torch, vd, path, w, peaks, barrier, args):
     for i in range(3):
         vd.vardrop_pearson_max(path.dev[i % slots]["x"], cfg, out, above, ws)
     vd.vardrop_profile_enable(True)
-    ms = time_region(torch, lambda i: vd.vardrop_pearson_max(path.dev[i % slots]["x"], cfg, out, above, ws), k, barrier)
+    t = time_region(torch, lambda i: vd.vardrop_pearson_max(path.dev[i % slots]["x"], cfg, out, above, ws), k, barrier)
     per = vd.vardrop_profile_read()
     vd.vardrop_profile_enable(False)
-    if vd.ws_status(ws) != vd.OK:
+    if vd.vardrop_ws_status(ws) != vd.OK:
         raise RuntimeError("device status set by vardrop_pearson_max")
     flops = 2.0 * w.B * float(w.N) ** 2 * w.L
-    t_max = per["pearson_max_kernel"][0] / k * 1e-3
-    res = {"ms_per_call": ms / k, "normalize_us": per["pearson_normalize_kernel"][0] / k * 1e3, "max_kernel_us": t_max * 1e6,
+    t_max = per["pearson_max_kernel"][0] / per["pearson_max_kernel"][1] * 1e-3
+    res = {"ms_per_call": t["median"], "normalize_us": per["pearson_normalize_kernel"][0] / per["pearson_normalize_kernel"][1] * 1e3,
+           "max_kernel_us": t_max * 1e6,
            "algorithmic_flops": flops, "tflops": flops / t_max / 1e12, "frac_of_bf16_peak": flops / t_max / 1e12 / peaks["bf16_tflops"],
            "share_above_0.9": float(above.float().mean().item()) / w.N, "note": "timed with the per-kernel event timer armed"}
     if not args.no_cpu:
+        import oracle
         x1 = path.host[0][0][:1].numpy()
         t0 = time.perf_counter()
         oracle.pearson_max(x1)
         res["oracle_ms_per_instance"] = (time.perf_counter() - t0) * 1e3
         res["oracle_cores"] = oracle.num_threads()
     return res
+
+
+def per_launch(per_kernel):
+    """{kernel: (total ms, launches)} -> the same with zero-launch kernels dropped."""
+    return {k: v for k, v in per_kernel.items() if v[1] > 0}
+
+
+def measure_off(torch, vd, path, w, peaks, barrier, steps):
+    """VarDrop off: the same attention kernels on all N tokens (the paper's inference / ground configuration), timed with
+    the per-kernel event timer armed."""
+    slots = len(path.dev)
+    for i in range(3):
+        path.step(i % slots, vardrop=False)
+    vd.vardrop_profile_enable(True)
+    t = time_region(torch, lambda i: path.step(i % slots, vardrop=False), steps, barrier, min_seconds=0.15, min_intervals=20)
+    pk = per_launch(vd.vardrop_profile_read())
+    vd.vardrop_profile_enable(False)
+    fwd_ms = pk["attn_fwd_kernel"][0] / pk["attn_fwd_kernel"][1]
+    bwd_ms = pk["attn_bwd_kernel"][0] / pk["attn_bwd_kernel"][1]
+    fl_f, fl_b = 4.0 * w.B * w.H * float(w.N) ** 2 * w.D, 10.0 * w.B * w.H * float(w.N) ** 2 * w.D
+    tf = (fl_f + fl_b) / ((fwd_ms + bwd_ms) * 1e-3) / 1e12
+    return {"ms_per_step": t["median"], "tokens_per_s": w.tokens / (t["median"] * 1e-3), "n_tokens": w.N,
+            "attn_fwd_ms": fwd_ms, "attn_bwd_ms": bwd_ms,
+            "attn_fwd_tflops": fl_f / (fwd_ms * 1e-3) / 1e12, "attn_bwd_tflops": fl_b / (bwd_ms * 1e-3) / 1e12,
+            "attn_tflops": tf, "attn_frac_of_bf16_peak": tf / peaks["bf16_tflops"],
+            "attn_frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+            "kernels": kernel_table(pk, kernel_work(w, w.N, selected=False), peaks),
+            "note": "attention kernels timed by CUDA events around every launch (timer armed)"}
+
+
+def traffic_targets(torch, vd, inputs, dist_util, device, rank, peaks, barrier, main_w, main_path, main_kernels, main_off):
+    """The figures the throughput targets are stated on, from a short pass over the Traffic-shaped workload (N = 862): all-token
+    attention forward + backward against the dense bf16 peak, and the k-DFH, selection and gather kernels against the HBM
+    peak.  When the main workload is Traffic itself its own tables are reused."""
+    if main_w.name == "traffic":
+        kernels, off = main_kernels, main_off
+    else:
+        w = inputs.WORKLOADS["traffic"]
+        path = Path(w, device, seed=dist_util.rank_seed(w.seed, rank), slots=8, host_slots=0)
+        slots = len(path.dev)
+        for i in range(5):
+            path.step(i % slots)
+        torch.cuda.synchronize()
+        n_sel = int(path.sel["n_sel"].item())
+        vd.vardrop_profile_enable(True)
+        time_region(torch, lambda i: path.step(i % slots), 50, barrier, min_seconds=0.05, min_intervals=20)
+        kernels = kernel_table(per_launch(vd.vardrop_profile_read()), kernel_work(w, n_sel), peaks)
+        vd.vardrop_profile_enable(False)
+        off = measure_off(torch, vd, path, w, peaks, barrier, 20)
+        path.check_status()
+        del path
+        torch.cuda.empty_cache()
+    if off is None:
+        return None
+    pick = lambda name: ({"avg_us": kernels[name]["avg_us"], "frac_of_hbm_peak": kernels[name]["frac"]} if name in kernels else None)
+    return {"workload": "traffic: B=32 N=862 L=96 k=3 rate=0.2 H=8 D=64",
+            "n862_attn_fwd_us": off["attn_fwd_ms"] * 1e3, "n862_attn_bwd_us": off["attn_bwd_ms"] * 1e3,
+            "n862_attn_tflops": off["attn_tflops"], "n862_attn_frac_of_bf16_peak": off["attn_frac_of_bf16_peak"],
+            "n862_attn_target_frac": 0.5,
+            "hash": pick("hash_kernel"), "select": pick("select_small_kernel"), "gather": pick("gather_kernel"),
+            "hbm_target_frac": 0.6,
+            "note": "per-kernel durations by CUDA events around every launch; fractions use algorithmic bytes / flops and the measured peaks"}
 
 
 def run_gpu(args):
@@ -323,75 +467,72 @@ def run_gpu(args):
     path.check_status()
     n_sel = int(path.sel["n_sel"].item())
     n_groups = int(path.sel["n_groups"].item())
+    gpu_keys = path.keys.cpu().numpy().view(np.uint64).copy()        # hash values of slot (warmup - 1) % slots, for the tie-flip count
+    keys_slot = (args.warmup - 1) % slots
 
-    # ---- timed region: K whole steps, device resident ---------------------------------------------------------
+    # ---- timed region: passes of K whole steps, device resident -----------------------------------------------
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
     launches0 = vd.vardrop_launch_count()
-    ms = time_region(torch, lambda i: path.step(i % slots), args.steps, barrier)
-    host_ms = time_region.host_ms
+    t_main = time_region(torch, lambda i: path.step(i % slots), args.steps, barrier)
     launches = vd.vardrop_launch_count() - launches0
-    # ---- same K steps with the per-kernel event timer armed (durations for the roofline) ----------------------
+    # ---- the same steps with the per-kernel event timer armed (durations for the roofline) --------------------
     vd.vardrop_profile_enable(True)
-    ms_armed = time_region(torch, lambda i: path.step(i % slots), args.steps, barrier)
-    per_kernel = vd.vardrop_profile_read()
+    t_armed = time_region(torch, lambda i: path.step(i % slots), args.steps, barrier, min_seconds=0.15, min_intervals=20)
+    per_kernel = per_launch(vd.vardrop_profile_read())
     vd.vardrop_profile_enable(False)
     # ---- end to end: host buffers, copies inside the timed region ----------------------------------------------
-    for i in range(2):
-        path.step_e2e(i % slots)
-    ms_e2e = time_region(torch, lambda i: path.step_e2e(i % slots), args.steps, barrier)
-    # ---- VarDrop off: the same attention kernels on all N tokens ---------------------------------------------
-    off = None
-    if not args.no_off:
-        for i in range(3):
-            path.step(i % slots, vardrop=False)
-        k_off = max(3, min(args.steps, 20))
-        vd.vardrop_profile_enable(True)
-        ms_off = time_region(torch, lambda i: path.step(i % slots, vardrop=False), k_off, barrier)
-        pk_off = vd.vardrop_profile_read()
-        vd.vardrop_profile_enable(False)
-        fl = 14.0 * w.B * w.H * float(w.N) ** 2 * w.D
-        t_attn = (pk_off["attn_fwd_kernel"][0] + pk_off["attn_bwd_kernel"][0]) / k_off * 1e-3
-        off = {"ms_per_step": ms_off / k_off, "tokens_per_s": w.tokens / (ms_off / k_off * 1e-3), "n_tokens": w.N,
-               "attn_fwd_ms": pk_off["attn_fwd_kernel"][0] / k_off, "attn_bwd_ms": pk_off["attn_bwd_kernel"][0] / k_off,
-               "attn_tflops": fl / t_attn / 1e12, "attn_frac_of_bf16_peak": fl / t_attn / 1e12 / peaks["bf16_tflops"],
-               "kernels": kernel_table(pk_off, kernel_work(w, w.N, selected=False), peaks),
-               "note": "timed with the per-kernel event timer armed"}
-    pearson = pearson_leg(torch, vd, path, w, peaks, barrier, args) if args.pearson else None
+    path.e2e_setup()
+    for i in range(3):
+        path.step_e2e(i)
+    torch.cuda.synchronize()
+    t_e2e = time_region(torch, path.step_e2e, args.steps, barrier, begin=path.e2e_begin, drain=path.e2e_drain)
     clocks = sampler.stop() if rank == 0 else None
+    # ---- VarDrop off, the target figures at N = 862, the redundancy check ---------------------------------------
+    off = None if args.no_off else measure_off(torch, vd, path, w, peaks, barrier, max(3, min(args.steps, 20)))
+    kernels = kernel_table(per_kernel, kernel_work(w, n_sel), peaks)
+    targets = None
+    if not args.no_targets and rank == 0 and world == 1:
+        targets = traffic_targets(torch, vd, inputs, dist_util, device, rank, peaks, barrier, w, path, kernels, off)
+    pearson = pearson_leg(torch, vd, path, w, peaks, barrier, args) if args.pearson else None
     path.check_status()
 
-    ms, ms_e2e = dist_util.max_over_ranks([ms, ms_e2e], dist, device)
+    ms, ms_mean, ms_e2e = dist_util.max_over_ranks([t_main["median"], t_main["mean"], t_e2e["median"]], dist, device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     tokens = w.tokens * world
-    kernels = kernel_table(per_kernel, kernel_work(w, n_sel), peaks)
     top = max(kernels, key=lambda k: kernels[k]["share"])
     roofline = {"kernel": top, "bound": kernels[top]["bound"], "achieved": kernels[top]["achieved"], "peak": kernels[top]["peak"],
                 "unit": kernels[top]["unit"], "frac": kernels[top]["frac"], "traffic": recorded_traffic(top, w.name),
                 "peak_source": f"{peak_kind} (burst figure for tensor work)",
-                "timing": "CUDA events around every launch, second pass of the same K steps",
-                "ms_per_step_with_timer_armed": ms_armed / args.steps}
+                "timing": "CUDA events around every launch, separate passes of the same K steps",
+                "ms_per_step_with_timer_armed": t_armed["median"]}
 
-    cpu = None if args.no_cpu else cpu_baseline(w, reps=2)
+    cpu, ties = (None, None) if args.no_cpu else cpu_baseline(w, reps=2, gpu_keys=gpu_keys, keys_x=path.host_x(keys_slot))
     line = {
-        "metric": METRIC, "value": dist_util.aggregate_throughput(w.tokens, world, ms / args.steps * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": dist_util.aggregate_throughput(w.tokens, world, ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "host_issue_ms_per_step": host_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_mean": ms_mean, "host_issue_ms_per_step": t_main["host_ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 attention (fp32 accumulate), fp32 FFT, integer grouping", "data": "synthetic",
         "config": {"workload": f"{w.name}: B={w.B} N={w.N} L={w.L} k={w.k} rate={w.rate} H={w.H} D={w.D}",
                    "kept_tokens": n_sel, "groups": n_groups, "delta": 1.0 - n_sel / w.N,
+                   "tie_flips": ties,
                    "l2": f"inputs and outputs rotate through {slots} sets ({slots * set_bytes / 2 ** 20:.0f} MiB > 126 MiB L2)",
                    "parallelism": f"dp{world} (independent batches per rank, no collective)"},
-        "clocks": clocks, "gpu_launches": launches,
-        "e2e": {"value": tokens / (ms_e2e / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": path.input_bytes(),
-                "d2h_bytes_per_step": path.output_bytes(), "ms_per_step": ms_e2e / args.steps},
-        "roofline": roofline, "kernels": kernels, "vardrop_off": off, "cpu_baseline": cpu,
+        "timing": {"statistic": "median of per-block CUDA-event intervals (a block is max(1, K // 64) steps); passes of exactly K steps "
+                                f"repeated until {MIN_REGION_S} s and {MIN_INTERVALS} intervals; max over ranks",
+                   "intervals": t_main["intervals"], "passes": t_main["passes"], "timed_ms_total": t_main["total_ms"]},
+        "clocks": clocks, "gpu_launches": launches, "gpu_launches_per_step": launches / (t_main["passes"] * args.steps),
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": path.input_bytes(),
+                "d2h_bytes_per_step": path.output_bytes(), "ms_per_step": ms_e2e,
+                "pipeline": "copies on two extra streams beside the kernels, two slots in rotation; every step copies all its inputs in and all its outputs out"},
+        "roofline": roofline, "kernels": kernels, "vardrop_off": off, "targets": targets, "cpu_baseline": cpu,
     }
     if pearson is not None:
         line["pearson"] = pearson
@@ -452,15 +593,25 @@ def sample_text(w, plan):
             f"the batch; grouping and sampling on all {w.N} variates")
 
 
-def cpu_baseline(w, reps):
+def cpu_baseline(w, reps, gpu_keys=None, keys_x=None):
+    """The oracle as it stands, timed on a bounded sample (see sample_text).  With `gpu_keys` (the hash values the CUDA path
+    produced for the windows `keys_x`) it also hashes that whole batch once and counts the variates whose hash differs: ties
+    the fp32 transform decides the other way on unfiltered inputs, and how many of those lie inside the 1e-3 relative gap."""
     import oracle
     x, toks = oracle_inputs(w)
     plan = oracle_plan(w, seconds_per_step=5.0)
     oracle_step(w, x, toks, 0, plan)
     secs = [oracle_step(w, x, toks, 1 + r, plan) for r in range(reps)]
     s = float(np.mean(secs))
+    ties = None
+    if gpu_keys is not None:
+        okeys, _, abar = oracle.hash(keys_x, w.k)
+        differ = okeys[0] != gpu_keys[0]
+        inside = oracle.rank_gaps(abar, w.k)[0] <= 1e-3
+        ties = {"variates": int(w.N), "hash_differs": int(differ.sum()), "of_which_inside_1e-3_gap": int((differ & inside).sum()),
+                "variates_inside_1e-3_gap": int(inside.sum())}
     return {"value": w.tokens / s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": sample_text(w, plan) + f"; mean of {reps} passes", "seconds_per_step": s}
+            "sample": sample_text(w, plan) + f"; mean of {reps} passes", "seconds_per_step": s}, ties
 
 
 def run_reference(args):
@@ -492,14 +643,20 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="elec", choices=["tiny", "elec", "traffic", "long", "scale"])
+    ap.add_argument("--workload", default="scale", choices=["tiny", "elec", "traffic", "long", "scale"],
+                    help="default: the largest single-GPU configuration")
     ap.add_argument("--impl", default="vardrop", choices=["vardrop", "reference"])
     ap.add_argument("--no-off", action="store_true", help="skip the VarDrop-off comparison pass")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline (profiling runs)")
+    ap.add_argument("--single-pass", action="store_true", help="one pass of K steps per timed region, no repetition (for ncu captures)")
+    ap.add_argument("--no-targets", action="store_true", help="skip the short Traffic-shaped pass behind the `targets` block")
     ap.add_argument("--pearson", action="store_true", help="also time the variate-redundancy check (Appendix A, Eq. 4) on the workload's windows")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.single_pass:
+        global MIN_REGION_S, MIN_INTERVALS
+        MIN_REGION_S, MIN_INTERVALS = 0.0, 1
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -54,6 +54,11 @@ const char* vardrop_status_string(int status);
 const char* vardrop_last_error(void);
 /* Library version, "major.minor". */
 const char* vardrop_version(void);
+/* Reads the device status word at the head of workspace `ws` (see "Problems found on the device" above): queues a
+ * 4-byte device-to-host copy on `stream`, waits for that stream, and returns the vardrop_status found there
+ * (VARDROP_ERR_CUDA when the copy itself fails).  This is the one entry point that synchronises; it never clears
+ * the word. */
+int vardrop_ws_status(const void* ws, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Measurement aids (no counterpart in the paper).
@@ -153,8 +158,9 @@ int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t*
  *
  * Same arguments, outputs and results as vardrop_select, minus ws / ws_bytes.
  * Limit: S * N <= 16384; larger problems return VARDROP_ERR_UNSUPPORTED (use vardrop_select).
- * It never calls cudaMalloc, cudaFree or any allocating routine; it issues one cudaMemsetAsync and
- * two kernel launches on `stream`.
+ * It never calls cudaMalloc, cudaFree or any allocating routine.  For N <= 2048 it issues one kernel launch
+ * and the built-in array is not touched; for larger N it issues one cudaMemsetAsync and three kernel
+ * launches on `stream`, all working in that array.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
  * device current) and caches it; make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps whatever the previous call left: the parts
@@ -208,8 +214,8 @@ int vardrop_attn_fwd(const void* q, const void* k, const void* v, const int32_t*
  * d_o         [B, N, H, D] bf16, gradient of o; rows 0..n_sel-1 are read.
  * inv_idx     [S, N] int32 from vardrop_select (NULL when sel_idx is NULL).
  * dq, dk, dv  [B, N, H, D] bf16 out, full variate layout.
- * dQ' is accumulated across key tiles with fp32 atomic adds, so its low-order bits may differ from run
- * to run; dK', dV' are bit-reproducible.
+ * With more than two key tiles dQ' is accumulated across key tiles by bulk fp32 reduce-adds that land in no fixed
+ * order, so the low-order bits of dq may differ from run to run; dK', dV' are bit-reproducible.
  * ---------------------------------------------------------------------------------------------- */
 int vardrop_attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
                      const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg* cfg,

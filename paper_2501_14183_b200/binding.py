@@ -44,7 +44,7 @@ class VardropError(RuntimeError):
         super().__init__(f"{where}: {lib.vardrop_status_string(status).decode()} ({status}): {lib.vardrop_last_error().decode()}")
 
 
-EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_hash_workspace_bytes", "vardrop_hash",
+EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_ws_status", "vardrop_hash_workspace_bytes", "vardrop_hash",
            "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_select_static", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
            "vardrop_attn_bwd", "vardrop_pearson_workspace_bytes", "vardrop_pearson_max", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
            "vardrop_profile_kernel_name", "vardrop_profile_read")
@@ -64,6 +64,8 @@ def load() -> C.CDLL:
                      "vardrop_pearson_workspace_bytes"):
             getattr(lib, name).restype = C.c_size_t
             getattr(lib, name).argtypes = [C.c_void_p]
+        lib.vardrop_ws_status.restype = C.c_int
+        lib.vardrop_ws_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.vardrop_hash.restype = C.c_int
         lib.vardrop_hash.argtypes = [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
         lib.vardrop_select.restype = C.c_int
@@ -176,9 +178,12 @@ def vardrop_profile_read() -> dict:
     return out
 
 
-def ws_status(ws) -> int:
+def vardrop_ws_status(ws) -> int:
     """Device-side status word of a workspace (synchronises the current stream)."""
-    return int(ws.view(torch.uint8)[:4].view(torch.int32).item())
+    return int(load().vardrop_ws_status(_ptr(ws), _stream()))
+
+
+ws_status = vardrop_ws_status
 
 
 # ---- buffer helpers (allocation only) -----------------------------------------------------------------------

@@ -27,16 +27,33 @@ def needs_build() -> bool:
     return LIB.stat().st_mtime < newest
 
 
+def _headers_mtime() -> float:
+    return max(p.stat().st_mtime for p in list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.h")) + [HERE.parent / "include" / "vardrop.h"])
+
+
 def build(force: bool = False, verbose: bool = False) -> Path:
+    """Compiles every translation unit that is out of date (objects live in _build/, compiled side by side) and links
+    the shared object."""
     if not force and not needs_build():
         return LIB
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-shared",
-           "-Xcompiler", "-fPIC", "-o", str(tmp)]
+    from concurrent.futures import ThreadPoolExecutor
+    obj_dir = HERE / "_build"
+    obj_dir.mkdir(exist_ok=True)
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC"]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [str(CSRC / s) for s in SOURCES]
-    subprocess.check_call(cmd)
+        flags += ["-Xptxas", "-v"]
+    hdr = _headers_mtime()
+
+    def compile_one(name: str) -> Path:
+        src, obj = CSRC / name, obj_dir / (name + ".o")
+        if force or verbose or not obj.exists() or obj.stat().st_mtime < max(src.stat().st_mtime, hdr):
+            subprocess.check_call([_nvcc(), *flags, "-c", "-o", str(obj), str(src)])
+        return obj
+
+    with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
+    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *[str(o) for o in objs]])
     os.replace(tmp, LIB)
     return LIB
 

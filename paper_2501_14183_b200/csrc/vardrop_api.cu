@@ -95,6 +95,15 @@ const char* vardrop_status_string(int status) {
 const char* vardrop_last_error(void) { return g_last_error; }
 const char* vardrop_version(void) { return "0.1"; }
 
+int vardrop_ws_status(const void* ws, void* stream) {
+    if (!ws) return fail(VARDROP_ERR_INVALID_ARG, "ws is NULL");
+    int word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int st = check_cuda(cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s), "ws_status: copy")) return st;
+    if (int st = check_cuda(cudaStreamSynchronize(s), "ws_status: synchronize")) return st;
+    return word;
+}
+
 long long vardrop_launch_count(void) {
     std::lock_guard<std::mutex> lock(g_prof_mutex);
     return g_launches;
