@@ -2,8 +2,8 @@
 //
 // bwd_prep_kernel    Delta_i = sum_d dO'_id O'_id and a zero-filled staged copy of dO' (rows past n_sel may hold
 //                    anything in the caller's buffer).  The fp32 dQ' accumulator is cleared by the forward kernel.
-// attn_bwd_kernel    one persistent CTA per SM (384 threads: 256 workers, one issuing warp, three more warps that help
-//                    drain dQ) over (128-key tile, head, instance), looping over the query tiles.  Scores are
+// attn_bwd_kernel    one persistent CTA per SM (384 threads: 256 workers and a third warpgroup whose first thread issues
+//                    the products) over (128-key tile, head, instance), looping over the query tiles.  Scores are
 //                    formed transposed (S^T = K Q^T, dP^T = V dO^T) so that two workers own each key row of tensor
 //                    memory; P^T and dS^T are written to shared memory once and feed three tensor-core products:
 //                    dV += P^T dO, dK += dS^T Q (accumulated in tensor memory across the query loop) and
@@ -161,9 +161,6 @@ __device__ __forceinline__ uint64_t mul_pair(uint64_t a, uint64_t b) {
     return d;
 }
 
-// every lane of the warp waits; the result is the same in all of them
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)); }
-
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -214,17 +211,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     unsigned char* sdSt = sPt + 2 * kTileBytes;     // dS^T : same shape
     unsigned char* sDQ = sdSt + 2 * kTileBytes;     // dQ_i as fp32: panel `half` = head dimensions 32 half .. 32 half + 31, 128-byte swizzled rows
     if (sDQ + 2 * kTileBytes > smem_dyn + kBwdSmemBytes) {
+        chain_wait();
         if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
         return;
     }
 
-    // Warps 0-3 are the third warpgroup (warp 0 issues the products: the warp schedulers favour the oldest ready warp, and its
-    // short dependent chains sit on every worker's critical path); warps 4-11 are the 256 workers.
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int wt = tid - 128;                       // worker index 0 .. 255 (negative in the third warpgroup)
-    const int wwarp = wt >> 5;                      // worker warp 0 .. 7
-    const int row = wt & (kTile - 1);               // tensor-memory lane this worker reads
-    const int half = wt >> 7;                       // which 64-column half of the lane
+    const int row = tid & (kTile - 1);              // tensor-memory lane this thread reads
+    const int half = tid >> 7;                      // which 64-column half of the lane
     if (warp == 0) {
         tmem_alloc(tmem_slot, kBwdTmemCols);
         tmem_relinquish();
@@ -265,14 +259,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int total_rows = P.B * P.N;
         const int lane = threadIdx.x & 31;
         const int warps_grid = gridDim.x * (kBwdWorkers >> 5);
-        const int wwarp = (static_cast<int>(threadIdx.x) >> 5) - 4;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
         uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
         uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
         uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
         int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
         while (group < 32 && group * warps_grid < total_rows) group <<= 1;
-        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + wwarp) * group; base < total_rows; base += warps_grid * group) {
+        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
             const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
             bool dropped = false;
             if (lane < group && r < total_rows) {
@@ -323,35 +316,35 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const uint64_t dq_ = umma_desc_advance(d_q0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
-            tc_mma_bf16_w(tm_st, umma_desc_advance(d_k, ks * 32), umma_desc_advance(dq_, ks * 32), idesc_kk, ks > 0);
-        tc_commit_w(bar_s);
+            tc_mma_bf16(tm_st, umma_desc_advance(d_k, ks * 32), umma_desc_advance(dq_, ks * 32), idesc_kk, ks > 0);
+        tc_commit(bar_s);
     };
     auto issue_dpt = [&](uint32_t stage) {
         const uint64_t dd_ = umma_desc_advance(d_do0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kDP / 16; ++ks)
-            tc_mma_bf16_w(tm_dpt, umma_desc_advance(d_v, ks * 32), umma_desc_advance(dd_, ks * 32), idesc_kk, ks > 0);
-        tc_commit_w(bar_dp);
+            tc_mma_bf16(tm_dpt, umma_desc_advance(d_v, ks * 32), umma_desc_advance(dd_, ks * 32), idesc_kk, ks > 0);
+        tc_commit(bar_dp);
     };
     auto issue_dv = [&](uint32_t stage, uint32_t acc_on) {           // reduction over the 128 queries
         const uint64_t mdo = umma_desc_advance(m_do0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kTile / 16; ++ks)
-            tc_mma_bf16_w(tm_dv, umma_desc_advance(d_pt, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mdo, ks * 2048), idesc_kmn,
+            tc_mma_bf16(tm_dv, umma_desc_advance(d_pt, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mdo, ks * 2048), idesc_kmn,
                         ks > 0 ? 1u : acc_on);
     };
     auto issue_dk = [&](uint32_t stage, uint32_t acc_on) {
         const uint64_t mq = umma_desc_advance(m_q0, stage * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kTile / 16; ++ks)
-            tc_mma_bf16_w(tm_dk, umma_desc_advance(d_dst, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mq, ks * 2048), idesc_kmn,
+            tc_mma_bf16(tm_dk, umma_desc_advance(d_dst, (ks >> 2) * kTileBytes + (ks & 3) * 32), umma_desc_advance(mq, ks * 2048), idesc_kmn,
                         ks > 0 ? 1u : acc_on);
     };
     auto issue_dq = [&]() {                                           // reduction over the 128 keys
 #pragma unroll
         for (int ks = 0; ks < kTile / 16; ++ks)
-            tc_mma_bf16_w(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
-        tc_commit_w(bar_g);
+            tc_mma_bf16(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
+        tc_commit(bar_g);
     };
 
     // minus the lse of query `qrow` in the log2 domain (fetched by the threads of half 0; -inf switches a missing query off)
@@ -377,16 +370,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         return a0.x * g0.x + a0.y * g0.y + a1.x * g1.x + a1.y * g1.y + a2.x * g2.x + a2.y * g2.y + a3.x * g3.x + a3.y * g3.y;
     };
 
-    if (warp < 4) {
+    if (warp >= kBwdWorkers / 32) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kBwdIssuerRegs));
         // The third warpgroup.  Its first thread queues the products as their operands become ready: the workers announce P^T
         // and dS^T on bar_p / bar_ds; the tensor core runs dV and the next S^T while they compute dS^T, and dQ, dK and the next
         // dP^T while they compute the next P^T.  All four warps (one per quarter of the tensor-memory lanes) then take dQ of the
         // tile out of tensor memory into the fp32 shared-memory tile, which one bulk reduction adds to the accumulator.
-        const bool iwarp = warp == 0;                   // the issuing warp: every lane runs the issue code (operands stay in uniform
-                                                        // registers), an elected lane executes each product
-        const bool issuer = tid == 0;                   // the one thread that owns the bulk reductions of dQ
-        const int qrow_l = tid;                         // query row this thread drains
+        const bool issuer = tid == kBwdWorkers;
+        const int qrow_l = tid - kBwdWorkers;           // query row this thread drains
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int jt = item % n_t_max;
             const int h = (item / n_t_max) % P.H;
@@ -395,32 +386,33 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             const int n_q = (kept + kTile - 1) / kTile;
             if (jt >= n_q) continue;
             const bool single_tile = n_q == 1;
-            if (iwarp) {
+            if (issuer) {
                 const uint32_t st0 = q_count % kQStages;
-                ok &= warp_wait(bar_kv, n_done & 1);
-                ok &= warp_wait(bar_qdo + st0, (q_count / kQStages) & 1);
+                ok &= mbar_wait(bar_kv, n_done & 1);
+                ok &= mbar_wait(bar_qdo + st0, (q_count / kQStages) & 1);
                 tc_fence_after();
                 issue_st(st0);
                 issue_dpt(st0);
             }
             for (int i = 0; i < n_q; ++i) {
                 const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
-                if (iwarp) {
-                    ok &= warp_wait(bar_p, ph);
+                if (issuer) {
+                    ok &= mbar_wait(bar_p, ph);
                     tc_fence_after();
                     issue_dv(st, i > 0);
                     if (i + 1 < n_q) {                   // S^T of the next query tile queues up behind dV
-                        ok &= warp_wait(bar_qdo + st1, ((qc + 1) / kQStages) & 1);
+                        ok &= mbar_wait(bar_qdo + st1, ((qc + 1) / kQStages) & 1);
                         tc_fence_after();
                         issue_st(st1);
                     }
-                    ok &= warp_wait(bar_ds, ph);
+                    ok &= mbar_wait(bar_ds, ph);
                     tc_fence_after();
                     issue_dq();
                     issue_dk(st, i > 0);
                     if (i + 1 < n_q) issue_dpt(st1);     // Q, dO of the next tile arrived before its S^T was issued
-                    else tc_commit_w(bar_acc);
+                    else tc_commit(bar_acc);
                 }
+                __syncwarp();                            // the issuer's warp waits for it here instead of polling beside it
                 if (!single_tile) {                      // (a single key tile: the workers write dQ with dV and dK at the end)
                     ok &= mbar_wait(bar_g, ph);
                     tc_fence_after();
@@ -461,7 +453,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             q_count += n_q;
             ++n_done;
         }
-        if (issuer) bulk_wait_group0();                  // the last dQ reductions have landed
+        if (tid == kBwdWorkers) bulk_wait_group0();      // the last dQ reductions have landed
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kBwdWorkerRegs));
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
@@ -480,10 +472,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         // Query tile i of this item rides ring stage (q_count at item start + i) mod 3; the k-th use of a stage completes
         // phase k of its barrier.  Tiles are fetched two ahead of the one being processed.
         auto fetch_qdo = [&](int i, uint32_t stage) {    // warps 2 and 3 fetch Q and dO of query tile i; one thread announces the bytes
-            if (wwarp == 2) {
+            if (warp == 2) {
                 if ((tid & 31) == 0) mbar_expect_tx(bar_qdo + stage, 2 * kTileBytes);
                 load_tile(sQ + stage * kTileBytes, &map_q, bar_qdo + stage, src, i * kTile, n_sel, h, b, P.H);
-            } else if (wwarp == 3) {
+            } else if (warp == 3) {
                 load_tile(sdO + stage * kTileBytes, &map_do, bar_qdo + stage, src_do, i * kTile, n_sel, h, b, P.H);
             }
         };
@@ -501,9 +493,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         {   // every MMA of the previous item has completed: K, V and every Q/dO stage are free.  Warps 0 .. 3 fetch K, V, Q, dO
             // side by side (each looks up its own gather rows); a barrier phase cannot complete before the thread that
             // announces its bytes has arrived, whichever comes first.
-            if (wt == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
-            if (wwarp == 0) load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            else if (wwarp == 1) load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            if (tid == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
+            if (warp == 0) load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
+            else if (warp == 1) load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
             fetch_qdo(0, st0);
             if (n_q > 1) fetch_qdo(1, (st0 + 1) % kQStages);
         }
@@ -652,9 +644,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (half == 0) s_nout[row] = key_valid ? n_out : -1;
             tc_fence_before();
             ok = worker_sync_and(ok);                    // the workers go on (or give up) together
-            const int c = wt & 7;
+            const int c = tid & 7;
             if (ok && c * 8 < P.D) {
-                for (int r = wt >> 3; r < kTile; r += kBwdWorkers / 8) {
+                for (int r = tid >> 3; r < kTile; r += kBwdWorkers / 8) {
                     const int n = s_nout[r];
                     if (n < 0) continue;
                     const size_t out = ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + c * 8;
@@ -673,7 +665,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (*flag) {
                 __threadfence();
                 const int chunks_head = P.D / 8;         // 16-byte output chunks per row
-                for (int idx = wt; idx < n_sel * chunks_head; idx += kBwdWorkers) {
+                for (int idx = tid; idx < n_sel * chunks_head; idx += kBwdWorkers) {
                     const int j = idx / chunks_head, dc = idx - j * chunks_head;
                     const float4* acc = reinterpret_cast<const float4*>(P.dq_acc + ((static_cast<size_t>(b) * P.Ncap + j) * P.H + h) * kDP) + dc * 2;
                     const float4 a0 = __ldcg(acc), a1 = __ldcg(acc + 1);
@@ -688,7 +680,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         ++n_done;
     }
     }   // workers
-    if (!zeros_written && wt >= 0) write_zero_rows();           // every item of this CTA was skipped (short instances)
+    if (!zeros_written && tid < kBwdWorkers) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();

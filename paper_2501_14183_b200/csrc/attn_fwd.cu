@@ -248,6 +248,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 
 // every lane of the warp waits; the result is the same in all of them
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)); }
+// the same with a sleep between polls: for warps whose reaction time is not on the critical path
+__device__ __forceinline__ bool warp_wait_relaxed(uint64_t* bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_relaxed(bar, parity)); }
 
 __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                    const __grid_constant__ CUtensorMap map_k,
@@ -337,14 +339,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             if (it.n_act <= 0) continue;
             TileSource src = P.src;
             if (src.idx) src.idx += static_cast<size_t>(P.S > 1 ? it.b : 0) * P.N;
-            ok = warp_wait(bar_q_free, (n_done & 1) ^ 1);
+            ok = warp_wait_relaxed(bar_q_free, (n_done & 1) ^ 1);
             if (!ok) break;
             if (lane == 0) mbar_expect_tx(bar_q_full, it.n_act * kTileBytes);
             for (int w = 0; w < it.n_act; ++w)
                 load_tile(sQ + w * kTileBytes, &map_q, bar_q_full, src, (kFwdGroups * it.p + w) * kTile, it.n_sel, it.h, it.b, P.H);
             for (int j = 0; j < it.n_kv; ++j, ++kv_iter) {
                 const uint32_t st = kv_iter % kFwdStages;
-                ok = warp_wait(bar_kv_free + st, ((kv_iter / kFwdStages) & 1) ^ 1);
+                ok = warp_wait_relaxed(bar_kv_free + st, ((kv_iter / kFwdStages) & 1) ^ 1);
                 if (!ok) break;
                 if (lane == 0) mbar_expect_tx(bar_kv_full + st, 2 * kTileBytes);
                 load_tile(sK + st * 2 * kTileBytes, &map_k, bar_kv_full + st, src, j * kTile, it.n_sel, it.h, it.b, P.H);
@@ -450,7 +452,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             }
             float m_ref = -INFINITY, l_run = 0.f;       // exponentials are taken against m_ref (log2 domain), which trails the running maximum
             for (int g = 0; g < it.n_half; ++g, ++t_cnt) {
-                ok = warp_wait(bar_s + w, t_cnt & 1);
+                ok = warp_wait_relaxed(bar_s + w, t_cnt & 1);
                 if (!ok) break;
                 tc_fence_after();
                 const int valid = min(kHalf, it.n_sel - g * kHalf);      // keys of this step that exist
@@ -525,7 +527,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             }
             if (!ok) break;
             // ---- epilogue: O / l, rounded to bf16, through a staging tile so that whole 128-byte rows are written -------------
-            ok = warp_wait(bar_o + w, n_done & 1);
+            ok = warp_wait_relaxed(bar_o + w, n_done & 1);
             if (!ok) break;
             tc_fence_after();
             {
@@ -547,7 +549,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             }
             tc_fence_before();
             mbar_arrive(bar_e + w);
-            ok = warp_wait(bar_e + w, n_done & 1);
+            ok = warp_wait_relaxed(bar_e + w, n_done & 1);
             if (!ok) break;
             {
                 const int c = r & 7;

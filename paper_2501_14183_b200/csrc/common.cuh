@@ -102,6 +102,23 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     }
 }
 
+// The same for warps off the critical path: a failed poll is followed by a short sleep, so that a waiting warp leaves the
+// issue slots of its scheduler to the warps that work (a spinning warp issues a poll loop's instructions back to back).
+#ifndef VD_SLEEP_NS
+#define VD_SLEEP_NS 32
+#endif
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        for (int it = 0; it < 64; ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if (VD_SLEEP_NS > 0) __nanosleep(VD_SLEEP_NS);
+        }
+        if (global_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
 // ---- TMA (bulk tensor copies) ----------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const void* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");

@@ -6,7 +6,7 @@
 // and is summed in ascending instance order.  Two real windows ride one complex transform
 // (z = x1 + i x2; X1_f = (Z_f + conj Z_{L-f}) / 2, X2_f = (Z_f - conj Z_{L-f}) / 2i), which is evaluated by
 // a Stockham autosort mixed-radix FFT (radices 4, 2, 3, 5, 7; larger prime factors as plain sums) whose butterflies are spread over the
-// whole CTA.  Twiddles are produced once per CTA in double precision.
+// whole CTA.  Twiddles are produced once per CTA with sincospif on an angle reduced to half a turn with integers.
 #include "common.cuh"
 #include "kernels.h"
 

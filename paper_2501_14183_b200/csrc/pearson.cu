@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(kPearsonThreads, 2) pearson_max_kernel(const P
     unsigned char* sA = align_tiles(smem_dyn + 64 + kTile * sizeof(float));      // row tile: hi, then lo (16 KB each)
     unsigned char* sB = sA + 2 * kTileBytes;                                     // column tile: hi, then lo (32 KB each)
     if (sB + 4 * kTileBytes > smem_dyn + kPearsonSmemBytes) {    // dynamic shared memory base not 1024-byte aligned
+        chain_wait();
         if (threadIdx.x == 0) set_status(P.status, VARDROP_ERR_CUDA);
         return;
     }
