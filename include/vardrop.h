@@ -60,6 +60,13 @@ const char* vardrop_version(void);
  * the word. */
 int vardrop_ws_status(const void* ws, void* stream);
 
+/* Failure-handling check (no counterpart in the paper).  Every wait inside the library's kernels is bounded: when it runs out the
+ * kernel records VARDROP_ERR_TIMEOUT in the status word and leaves through its normal exit, so the context stays usable.
+ * This call launches one warp that waits `limit_us` microseconds (1 .. 100000) on a barrier nothing ever completes, through
+ * that same wait, so that the path can be seen to work: afterwards vardrop_ws_status(ws) is VARDROP_ERR_TIMEOUT and later
+ * calls on the stream run normally.  ws: at least 256 bytes. */
+int vardrop_probe_bounded_wait(void* ws, size_t ws_bytes, unsigned int limit_us, void* stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Measurement aids (no counterpart in the paper).
  *   vardrop_launch_count          kernels this library has launched in this process so far.
@@ -171,6 +178,26 @@ int vardrop_select(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t*
 int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, int32_t* group_id, int32_t* group_offsets,
                           int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx,
                           void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Gather of the kept raw variates -- Sec. 3.3 ("Token Reduction"): the dropped variates are removed from the
+ * lookback window itself, before the embedding, so that every later layer works on N' variates:
+ *   x_sel[b, j, :] = x[b, sel_idx[s(b), j], :]   for j < n_sel[s(b)],   s(b) = 0 (S = 1) or b (S = B).
+ * A pure copy, bit-exact.
+ *
+ * cfg (host)  B, N, L shape of x; S = 1 (one selection for the batch) or B (one per instance).
+ * x           [B, N, L] float32, contiguous.
+ * sel_idx     [S, N] int32, n_sel [S] int32: vardrop_select's outputs.
+ * x_sel       [B, N, L] float32 out (capacity of all N variates); rows 0 .. n_sel-1 of instance b are written, the
+ *             rest is untouched.
+ * No workspace and no device status: nothing can go wrong on the device that the host did not check.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t B, N, L, S;
+} vardrop_gather_cfg;
+
+int vardrop_gather_rows(const float* x, const int32_t* sel_idx, const int32_t* n_sel, const vardrop_gather_cfg* cfg,
+                        float* x_sel, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Attention over the kept tokens -- Sec. 3.3 (token reduction: only the selected variate tokens enter

@@ -153,3 +153,15 @@ def pearson_max(x: np.ndarray) -> np.ndarray:
     _load().vdo_pearson_max(_p(x), B, N, L, _p(out))
     return out
 
+
+
+def gather_rows(x: np.ndarray, sel: np.ndarray, n_sel: np.ndarray, fill: float = 0.0) -> np.ndarray:
+    """Sec. 3.3 on the raw window: rows 0..n_sel-1 of instance b are x[b, sel[s(b), j], :]; the other rows keep ``fill``.
+    sel is [S, N] (S = 1 or B), n_sel [S]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    sel = np.ascontiguousarray(np.atleast_2d(sel), dtype=np.int32)
+    n_sel = np.ascontiguousarray(np.atleast_1d(n_sel), dtype=np.int32)
+    B, N, L = x.shape
+    out = np.full((B, N, L), fill, dtype=np.float32)
+    _load().vdo_gather_rows(_p(x), C.c_int(B), C.c_int(N), C.c_int(L), _p(sel), _p(n_sel), C.c_int(sel.shape[0]), _p(out))
+    return out

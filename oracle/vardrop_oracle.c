@@ -394,3 +394,18 @@ void vdo_pearson_max(const float* x, int B, int N, int L, double* max_rho) {
         }
     }
 }
+
+/* ---------------------------------------------------------------------------------------------------
+ * Token reduction on the raw window (Sec. 3.3): the kept variates of every instance, in the order of sel.
+ *   x      [B, N, L] float32
+ *   sel    [S, N] int32 (S = 1: one selection for the batch; S = B: one per instance), n_sel [S]
+ *   x_sel  [B, N, L] float32: rows 0 .. n_sel-1 of instance b are x[b, sel[s(b), j], :]; other rows are left alone
+ * ------------------------------------------------------------------------------------------------- */
+void vdo_gather_rows(const float* x, int B, int N, int L, const int32_t* sel, const int32_t* n_sel, int S, float* x_sel) {
+    for (int b = 0; b < B; ++b) {
+        const int s = S > 1 ? b : 0;
+        for (int j = 0; j < n_sel[s]; ++j)
+            for (int t = 0; t < L; ++t)
+                x_sel[((size_t)b * N + j) * L + t] = x[((size_t)b * N + sel[(size_t)s * N + j]) * L + t];
+    }
+}

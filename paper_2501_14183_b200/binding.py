@@ -33,6 +33,10 @@ class AttnCfg(C.Structure):
     _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float), ("S", C.c_int32)]
 
 
+class GatherCfg(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("L", C.c_int32), ("S", C.c_int32)]
+
+
 class PearsonCfg(C.Structure):
     _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("L", C.c_int32), ("threshold", C.c_float)]
 
@@ -44,8 +48,8 @@ class VardropError(RuntimeError):
         super().__init__(f"{where}: {lib.vardrop_status_string(status).decode()} ({status}): {lib.vardrop_last_error().decode()}")
 
 
-EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_ws_status", "vardrop_hash_workspace_bytes", "vardrop_hash",
-           "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_select_static", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
+EXPORTS = ("vardrop_status_string", "vardrop_last_error", "vardrop_version", "vardrop_ws_status", "vardrop_probe_bounded_wait", "vardrop_hash_workspace_bytes", "vardrop_hash",
+           "vardrop_select_workspace_bytes", "vardrop_select", "vardrop_select_static", "vardrop_gather_rows", "vardrop_attn_workspace_bytes", "vardrop_attn_fwd",
            "vardrop_attn_bwd", "vardrop_pearson_workspace_bytes", "vardrop_pearson_max", "vardrop_launch_count", "vardrop_profile_enable", "vardrop_profile_kernels",
            "vardrop_profile_kernel_name", "vardrop_profile_read")
 
@@ -66,12 +70,16 @@ def load() -> C.CDLL:
             getattr(lib, name).argtypes = [C.c_void_p]
         lib.vardrop_ws_status.restype = C.c_int
         lib.vardrop_ws_status.argtypes = [C.c_void_p, C.c_void_p]
+        lib.vardrop_probe_bounded_wait.restype = C.c_int
+        lib.vardrop_probe_bounded_wait.argtypes = [C.c_void_p, C.c_size_t, C.c_uint, C.c_void_p]
         lib.vardrop_hash.restype = C.c_int
         lib.vardrop_hash.argtypes = [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
         lib.vardrop_select.restype = C.c_int
         lib.vardrop_select.argtypes = [C.c_void_p] * 10 + [C.c_size_t, C.c_void_p]
         lib.vardrop_select_static.restype = C.c_int
         lib.vardrop_select_static.argtypes = [C.c_void_p] * 10
+        lib.vardrop_gather_rows.restype = C.c_int
+        lib.vardrop_gather_rows.argtypes = [C.c_void_p] * 6
         lib.vardrop_attn_fwd.restype = C.c_int
         lib.vardrop_attn_fwd.argtypes = [C.c_void_p] * 9 + [C.c_size_t, C.c_void_p]
         lib.vardrop_attn_bwd.restype = C.c_int
@@ -139,6 +147,10 @@ def vardrop_select_static(keys, cfg: SelectCfg, group_id, group_offsets, members
            "vardrop_select_static")
 
 
+def vardrop_gather_rows(x, sel_idx, n_sel, cfg: GatherCfg, x_sel) -> None:
+    _check(load().vardrop_gather_rows(_ptr(x), _ptr(sel_idx), _ptr(n_sel), C.byref(cfg), _ptr(x_sel), _stream()), "vardrop_gather_rows")
+
+
 def vardrop_attn_fwd(q, k, v, sel_idx, n_sel, cfg: AttnCfg, o, lse, ws) -> None:
     _check(load().vardrop_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(sel_idx), _ptr(n_sel), C.byref(cfg), _ptr(o), _ptr(lse),
                                    _ptr(ws), ws.numel() * ws.element_size(), _stream()), "vardrop_attn_fwd")
@@ -184,6 +196,10 @@ def vardrop_ws_status(ws) -> int:
 
 
 ws_status = vardrop_ws_status
+
+
+def vardrop_probe_bounded_wait(ws, limit_us: int) -> None:
+    _check(load().vardrop_probe_bounded_wait(_ptr(ws), ws.numel() * ws.element_size(), int(limit_us), _stream()), "vardrop_probe_bounded_wait")
 
 
 # ---- buffer helpers (allocation only) -----------------------------------------------------------------------

@@ -9,7 +9,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libvardrop.so"
-SOURCES = ["vardrop_api.cu", "hash.cu", "hash_rows.cu", "select.cu", "attn_fwd.cu", "attn_bwd.cu", "pearson.cu"]
+SOURCES = ["vardrop_api.cu", "hash.cu", "hash_rows.cu", "select.cu", "attn_fwd.cu", "attn_bwd.cu", "pearson.cu", "gather_rows.cu"]
 
 
 def _nvcc() -> str:

@@ -155,16 +155,36 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
     const int chunks_row = P.H * (kDP / 8);                                   // 16-byte chunks per staged token
     const int src_chunks_head = P.D / 8;
     const int total = n_fill * chunks_row;
-    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-        const int j = idx / chunks_row;
-        const int c = idx - j * chunks_row;
-        const int h = c / (kDP / 8), dc = c - h * (kDP / 8);
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (j < n_sel && dc < src_chunks_head) {
-            const int n = sel ? sel[j] : j;
-            val = __ldg(P.src[t] + (static_cast<size_t>(b) * P.N + n) * (P.H * src_chunks_head) + h * src_chunks_head + dc);
+    const uint4* src_b = P.src[t] + static_cast<size_t>(b) * P.N * (P.H * src_chunks_head);
+    uint4* dst_b = P.dst[t] + static_cast<size_t>(b) * P.Ncap * chunks_row;
+    // four chunks per thread and trip, a whole CTA apart, so that four independent row lookups and four 16-byte loads are in
+    // flight per thread before the first store (one load per trip leaves the memory system idle most of the time)
+    constexpr int U = 4;
+    const int stride = gridDim.x * blockDim.x;
+    for (int base = blockIdx.x * blockDim.x + threadIdx.x; base < total; base += U * stride) {
+        const uint4* from[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = base + u * stride;
+            from[u] = nullptr;
+            if (idx < total) {
+                const int j = idx / chunks_row;
+                const int c = idx - j * chunks_row;
+                const int h = c / (kDP / 8), dc = c - h * (kDP / 8);
+                if (j < n_sel && dc < src_chunks_head) {
+                    const int n = sel ? __ldg(sel + j) : j;
+                    from[u] = src_b + static_cast<size_t>(n) * (P.H * src_chunks_head) + h * src_chunks_head + dc;
+                }
+            }
         }
-        P.dst[t][(static_cast<size_t>(b) * P.Ncap + j) * chunks_row + c] = val;
+        uint4 val[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) val[u] = from[u] ? __ldg(from[u]) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = base + u * stride;
+            if (idx < total) dst_b[idx] = val[u];
+        }
     }
 }
 
@@ -846,7 +866,8 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D; G.S = attn_sel_rows(c);
         const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
         int gx = static_cast<int>((work + 255) / 256);
-        const int cap = max(1, 4 * sm_count() / (3 * c.B));        // about four CTAs per SM in total; each strides over its rows
+        const int cap = max(1, 8 * sm_count() / (3 * c.B));        // about eight CTAs per SM in total (the kept count is only known on the
+                                                                   // device: a grid sized for every variate would be mostly empty CTAs)
         if (gx > cap) gx = cap;
         cudaError_t gerr;
         { LaunchScope ls_(K_GATHER, stream); gerr = launch_chained(gather_kernel, dim3(gx, c.B, 3), dim3(256), 0, stream, G); }

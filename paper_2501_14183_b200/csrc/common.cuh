@@ -91,17 +91,17 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+constexpr uint64_t kWaitLimitNs = 2000000000ull;      // every wait of the library gives up after about two seconds
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
     for (int it = 0; it < 64; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (;;) {
         for (int it = 0; it < 256; ++it)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > 2000000000ull) return false;
+        if (global_ns() - t0 > limit_ns) return false;
     }
 }
-
 // The same for warps off the critical path: a failed poll is followed by a short sleep, so that a waiting warp leaves the
 // issue slots of its scheduler to the warps that work (a spinning warp issues a poll loop's instructions back to back).
 #ifndef VD_SLEEP_NS
@@ -115,7 +115,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
             if (mbar_try_wait(bar, parity)) return true;
             if (VD_SLEEP_NS > 0) __nanosleep(VD_SLEEP_NS);
         }
-        if (global_ns() - t0 > 2000000000ull) return false;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
     }
 }
 

@@ -11,7 +11,7 @@ namespace vardrop {
 
 // Kernel identities for the launch counter and the optional per-kernel event timer (vardrop_profile_*).
 enum KernelId {
-    K_HASH = 0, K_SELECT_SMALL, K_SELECT_COUNT, K_SELECT_GROUP, K_SELECT_SAMPLE, K_GATHER, K_ATTN_FWD, K_BWD_PREP, K_ATTN_BWD, K_BWD_CONVERT, K_PEARSON_NORM, K_PEARSON_MAX, K_COUNT
+    K_HASH = 0, K_SELECT_SMALL, K_SELECT_COUNT, K_SELECT_GROUP, K_SELECT_SAMPLE, K_GATHER, K_ATTN_FWD, K_BWD_PREP, K_ATTN_BWD, K_BWD_CONVERT, K_PEARSON_NORM, K_PEARSON_MAX, K_GATHER_ROWS, K_COUNT
 };
 // Wrap a kernel launch: counts it and, when the timer is armed, brackets it with a pair of CUDA events on `stream`.
 struct LaunchScope {
@@ -44,6 +44,10 @@ constexpr int kStaticMaxRows = 16384;                 // largest S * N it accept
 constexpr int kStaticSelectBytes = 400 * 1024;        // size of that array
 int select_static_launch(const uint64_t* keys, const vardrop_select_cfg& cfg, int32_t* group_id, int32_t* group_offsets,
                          int32_t* members, int32_t* n_groups, int32_t* sel_idx, int32_t* n_sel, int32_t* inv_idx, cudaStream_t stream);
+
+// gather_rows.cu
+int gather_rows_validate(const vardrop_gather_cfg& cfg);
+int gather_rows_launch(const float* x, const int32_t* sel_idx, const int32_t* n_sel, const vardrop_gather_cfg& cfg, float* x_sel, cudaStream_t stream);
 
 // pearson.cu
 size_t pearson_workspace_bytes(const vardrop_pearson_cfg& cfg);

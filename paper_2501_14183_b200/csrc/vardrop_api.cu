@@ -48,7 +48,7 @@ std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_events[K_COUNT];   // pa
 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_prof_free;              // pairs ready for reuse
 const char* const g_kernel_names[K_COUNT] = {"hash_kernel", "select_small_kernel", "select_count_kernel", "select_group_kernel", "select_sample_kernel", "gather_kernel",
                                              "attn_fwd_kernel", "bwd_prep_kernel", "attn_bwd_kernel", "bwd_convert_kernel", "pearson_normalize_kernel",
-                                             "pearson_max_kernel"};
+                                             "pearson_max_kernel", "gather_rows_kernel"};
 }  // namespace
 
 LaunchScope::LaunchScope(int id, cudaStream_t stream) : id_(id), stream_(stream), stop_(nullptr) {
@@ -69,6 +69,21 @@ LaunchScope::LaunchScope(int id, cudaStream_t stream) : id_(id), stream_(stream)
 
 LaunchScope::~LaunchScope() {
     if (stop_) cudaEventRecord(static_cast<cudaEvent_t>(stop_), stream_);
+}
+
+// A wait that nothing ever completes: one warp polls a fresh barrier with the library's bounded wait and a caller-chosen limit,
+// then reports the way every kernel of the library does (status word, normal exit).
+__global__ void bounded_wait_probe_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    chain_wait();
+    chain_release();
+    const bool done = mbar_wait(&bar, 0, limit_ns);
+    if (!__all_sync(0xffffffffu, done) && threadIdx.x == 0) set_status(status, VARDROP_ERR_TIMEOUT);
 }
 
 }  // namespace vardrop
@@ -102,6 +117,14 @@ int vardrop_ws_status(const void* ws, void* stream) {
     if (int st = check_cuda(cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s), "ws_status: copy")) return st;
     if (int st = check_cuda(cudaStreamSynchronize(s), "ws_status: synchronize")) return st;
     return word;
+}
+
+int vardrop_probe_bounded_wait(void* ws, size_t ws_bytes, unsigned int limit_us, void* stream) {
+    VD_CHECK(check_ws(ws, ws_bytes, kWsHeaderBytes));
+    if (limit_us < 1 || limit_us > 100000) return fail(VARDROP_ERR_INVALID_ARG, "probe: limit of %u us outside 1..100000", limit_us);
+    const cudaError_t err = launch_chained(bounded_wait_probe_kernel, dim3(1), dim3(32), 0, static_cast<cudaStream_t>(stream), static_cast<int*>(ws),
+                                           static_cast<unsigned long long>(limit_us) * 1000ull);
+    return check_cuda(err, "probe: launch");
 }
 
 long long vardrop_launch_count(void) {
@@ -191,6 +214,16 @@ int vardrop_select_static(const uint64_t* keys, const vardrop_select_cfg* cfg, i
     VD_CHECK(check_ptr(inv_idx, "inv_idx", true));
     return select_static_launch(keys, *cfg, group_id, group_offsets, members, n_groups, sel_idx, n_sel, inv_idx,
                                 static_cast<cudaStream_t>(stream));
+}
+
+int vardrop_gather_rows(const float* x, const int32_t* sel_idx, const int32_t* n_sel, const vardrop_gather_cfg* cfg, float* x_sel, void* stream) {
+    if (!cfg) return fail(VARDROP_ERR_INVALID_ARG, "cfg is NULL");
+    VD_CHECK(gather_rows_validate(*cfg));
+    VD_CHECK(check_ptr(x, "x", true));
+    VD_CHECK(check_ptr(sel_idx, "sel_idx", true));
+    VD_CHECK(check_ptr(n_sel, "n_sel", true));
+    VD_CHECK(check_ptr(x_sel, "x_sel", true));
+    return gather_rows_launch(x, sel_idx, n_sel, *cfg, x_sel, static_cast<cudaStream_t>(stream));
 }
 
 size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg) {

@@ -182,3 +182,24 @@ def test_back_to_back_steps_match_isolated_steps(name):
                 diff = torch.nan_to_num(diff, nan=1e9)
                 raise AssertionError(f"step {s} tensor {n}: {int((diff > 0).sum())} differing elements, max {float(diff.max()):.3e}, "
                                      f"first at {torch.nonzero(diff > 0)[0].tolist()}")
+
+
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """Failure handling without a fault: a warp waits 500 microseconds on a barrier nothing completes, through the bounded wait every
+    kernel uses; the status word then reads TIMEOUT, and a normal call on the same stream with a fresh status word still works."""
+    ws = vd.alloc_ws(4096)
+    vd.vardrop_probe_bounded_wait(ws, 500)
+    assert vd.vardrop_ws_status(ws) == vd.ERR_TIMEOUT
+    vd.vardrop_probe_bounded_wait(ws, 200)                      # the word is sticky: still the first problem
+    assert vd.vardrop_ws_status(ws) == vd.ERR_TIMEOUT
+    w = inputs.WORKLOADS["tiny"]
+    x = torch.from_numpy(inputs.make_windows(w)).cuda()
+    hcfg = vd.HashCfg(w.B, w.N, w.L, w.k, 0, 0, 0)
+    keys, freqs, _ = vd.alloc_hash_outputs(hcfg)
+    hws = vd.alloc_ws(vd.vardrop_hash_workspace_bytes(hcfg))
+    vd.vardrop_hash(x, hcfg, keys, freqs, None, hws)
+    assert vd.vardrop_ws_status(hws) == vd.OK
+    want, _, _ = oracle.hash(inputs.make_windows(w), w.k)
+    assert np.array_equal(keys.cpu().numpy().view(np.uint64), want)
+    with pytest.raises(vd.VardropError):
+        vd.vardrop_probe_bounded_wait(ws, 0)

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2501_14183_b200 import binding as vd
 from paper_2501_14183_b200 import inputs
 
@@ -33,14 +34,23 @@ def test_static_variant_matches_on_two_calls_in_a_row():
              (inputs.make_keys(862, 60, k=3, f_hi=25, seed=2), vd.SelectCfg(1, 862, 10, 1.0, 5, 8))]
     keys_t = [torch.from_numpy(k.reshape(1, -1).view(np.int64)).cuda() for k, _ in cases]
     outs = [vd.alloc_select_outputs(cfg) for _, cfg in cases]          # outputs are the caller's: allocated up front
+    torch.cuda.synchronize()
+    torch_before = torch.cuda.memory_allocated()
+    free_before, _ = torch.cuda.mem_get_info()
     for kt, (_, cfg), out in zip(keys_t, cases, outs):
         without_workspace(kt, cfg, out)                                # the two calls in a row, nothing in between
     torch.cuda.synchronize()
-    for kt, (_, cfg), out in zip(keys_t, cases, outs):
+    # the point of the variant: no device memory was obtained anywhere, neither through torch's allocator nor behind its back
+    assert torch.cuda.memory_allocated() == torch_before
+    assert torch.cuda.mem_get_info()[0] == free_before
+    for kt, (keys, cfg), out in zip(keys_t, cases, outs):
         want = with_workspace(kt, cfg)
         torch.cuda.synchronize()
         for name in NAMES:
             assert torch.equal(out[name], want[name]), name              # integer work: bit-exact
+        ref = oracle.select(keys.reshape(1, -1), cfg.gs, cfg.rate, cfg.seed, cfg.step)       # and pinned to the oracle, not only to its sibling
+        for name in NAMES:
+            assert np.array_equal(out[name].cpu().numpy(), ref[name]), name
 
 
 def test_static_variant_repeats_and_handles_several_hash_rows():
