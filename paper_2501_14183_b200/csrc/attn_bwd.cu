@@ -161,6 +161,11 @@ __device__ __forceinline__ uint64_t mul_pair(uint64_t a, uint64_t b) {
     return d;
 }
 
+// every lane of the warp waits; the result is the same in all of them
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)); }
+// the same with a sleep between polls: for warps whose reaction time is not on the critical path
+__device__ __forceinline__ bool warp_wait_relaxed(uint64_t* bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_relaxed(bar, parity)); }
+
 __device__ __forceinline__ float fast_exp2(float x) {      // special-function unit; exp2(-inf) = 0
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -688,6 +693,512 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// main, many tiles: the two phases of a (key tile, query tile) pair on warpgroups of their own
+// ---------------------------------------------------------------------------------------------------------
+// In the kernel above the same 256 threads turn S^T into P^T and then dP^T into dS^T, and the tensor core waits for each.
+// With many query tiles per key tile that serial worker time is the whole step, so this kernel gives each phase its own 256
+// threads and lets phase A of query tile i + 1 run beside phase B of tile i:
+//   warps 0-2    issue the products, each its own chain (all lanes run the issue code, an elected lane executes each product);
+//                warp 3 completes the register-donor warpgroup
+//   warps 4-11   phase A: P^T = exp2(S^T scale - lse), written to tensor memory as bf16 (the A operand of dV += P^T dO); they
+//                also take dQ of the previous tile out of tensor memory for the bulk reduce-add
+//   warps 12-19  phase B: dS^T = P^T o (dP^T - Delta) with P^T read back from tensor memory, written to tensor memory
+//                over the consumed columns of dP^T (the A operand of dK += dS^T Q) and to shared memory (dQ = dS K
+//                reads it transposed)
+// P^T and dS^T never pass through shared memory on their way to dV and dK, which takes 128 KB of shared-memory traffic
+// off every tile pair (shared-memory bandwidth, not the tensor pipe, bounds these products at a head dimension of 64).
+// Tensor memory: S^T [0,128) dP^T / dS^T [128,256) dV [256,320) dK [320,384) dQ [384,448) P^T [448,512).
+// Delta is always precomputed here (the host takes this kernel only where the prep kernel runs) and tiles arrive as
+// boxes (direct or staged).
+constexpr int kPipeThreads = 640;
+constexpr int kPipeGroup = 256;
+constexpr int kPipeSmallRegs = 64;     // launched with 640 x 96 = 61440 registers: 128 x 64 + 512 x 104
+constexpr int kPipeBigRegs = 104;
+constexpr int kPipeHeader = 4096;      // barriers, row statistics, scatter indices
+constexpr int kPipeSmemBytes = kPipeHeader + 2 * kTileBytes /*K, V*/ + 2 * kQStages * kTileBytes /*Q, dO ring*/ + 2 * kTileBytes /*dS^T*/ +
+                               2 * kTileBytes /*dQ tile, fp32, two 32-column halves*/;
+
+template <int kId>
+__device__ __forceinline__ bool group_sync_and(bool ok) {      // named barrier kId among 256 threads, and-reduction of ok
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "bar.red.and.pred p, %2, 256, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(ok)), "n"(kId)
+        : "memory");
+    return r != 0;
+}
+
+__global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                         const __grid_constant__ CUtensorMap map_k,
+                                                                         const __grid_constant__ CUtensorMap map_v,
+                                                                         const __grid_constant__ CUtensorMap map_do,
+                                                                         const __grid_constant__ CUtensorMap map_acc, const BwdParams P) {
+    extern __shared__ unsigned char smem_dyn[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_dyn);
+    uint64_t* bar_kv = bars + 0;
+    uint64_t* bar_qdo = bars + 1;                   // [3]
+    uint64_t* bar_s = bars + 4;                     // S^T of a query tile complete
+    uint64_t* bar_sfree = bars + 5;                 // phase A holds S^T in registers (256 arrivals): the next S^T may be produced
+    uint64_t* bar_p = bars + 6;                     // P^T in tensor memory (256 arrivals)
+    uint64_t* bar_pfree = bars + 7;                 // phase B holds P^T in registers (256 arrivals) and dV has read it (1 commit)
+    uint64_t* bar_dp = bars + 8;                    // dP^T of a query tile complete (and every product issued before it)
+    uint64_t* bar_ds = bars + 9;                    // dS^T in tensor and shared memory (256 arrivals)
+    uint64_t* bar_g = bars + 10;                    // dQ of a query tile complete
+    uint64_t* bar_acc = bars + 11;                  // every product of the item complete: dV, dK final, operands free
+    uint64_t* bar_dqfree = bars + 12;               // dQ of a query tile has left tensor memory (256 arrivals): the next one may be produced
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_dyn + 128);
+    int* s_scratch = reinterpret_cast<int*>(smem_dyn + 132);
+    float* s_stat = reinterpret_cast<float*>(smem_dyn + 256);     // [3 stages][128] minus the lse of the query tile, log2 domain
+    float* s_delta = s_stat + kQStages * kTile;                   // [2][128] Delta of the query tile, one array per tile parity
+    int* s_nout = reinterpret_cast<int*>(s_delta + 2 * kTile);    // [2][128] variate of each key row (-1: no such row), one array per item parity
+    unsigned char* sK = align_tiles(smem_dyn + 256 + (kQStages + 4) * kTile * sizeof(float));
+    unsigned char* sV = sK + kTileBytes;
+    unsigned char* sQ = sV + kTileBytes;               // 3 stages
+    unsigned char* sdO = sQ + kQStages * kTileBytes;   // 3 stages
+    unsigned char* sdSt = sdO + kQStages * kTileBytes; // dS^T : rows = keys, columns = queries (two 64-query panels); dV / dK staging at the end of an item
+    unsigned char* sDQ = sdSt + 2 * kTileBytes;        // dQ_i as fp32: panel `half` = head dimensions 32 half .. 32 half + 31, 128-byte swizzled rows
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (sDQ + 2 * kTileBytes > smem_dyn + kPipeSmemBytes) {
+        chain_wait();
+        if (tid == 0) set_status(P.status, VARDROP_ERR_CUDA);
+        return;
+    }
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, kBwdTmemCols);
+        tmem_relinquish();
+    }
+    if (tid == 0) {
+        mbar_init(bar_kv, 1);
+        for (int st = 0; st < kQStages; ++st) mbar_init(bar_qdo + st, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_sfree, kPipeGroup);
+        mbar_init(bar_p, kPipeGroup);
+        mbar_init(bar_pfree, kPipeGroup + 1);
+        mbar_init(bar_dp, 1);
+        mbar_init(bar_ds, kPipeGroup);
+        mbar_init(bar_g, 1);
+        mbar_init(bar_acc, 3);
+        mbar_init(bar_dqfree, kPipeGroup);
+        mbar_fence_init();
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+        tma_prefetch_desc(&map_do);
+        tma_prefetch_desc(&map_acc);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    chain_wait();
+    chain_release();
+    const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
+    const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, s_scratch) : kept_shared) + kTile - 1) / kTile;
+    const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
+
+    const uint32_t tm_st = tmem;            // [0,128)   S^T
+    const uint32_t tm_dpt = tmem + 128;     // [128,256) dP^T; dS^T (bf16) over its consumed columns: queries 64 half .. at column 64 half
+    const uint32_t tm_dv = tmem + 256;      // [256,320) dV
+    const uint32_t tm_dk = tmem + 320;      // [320,384) dK
+    const uint32_t tm_dq = tmem + 384;      // [384,448) dQ of the current query tile
+    const uint32_t tm_pt = tmem + 448;      // [448,512) P^T (bf16): queries 2 c, 2 c + 1 in column c
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    bool ok = true;
+    uint32_t q_count = 0;       // query tiles consumed so far by this CTA: ring stage = q_count mod 3
+    uint32_t n_done = 0;        // work items finished by this CTA
+
+    struct Item { int jt, h, b, n_sel, n_q; };
+    auto decode = [&](int item) {
+        Item it;
+        it.jt = item % n_t_max;
+        it.h = (item / n_t_max) % P.H;
+        it.b = item / (n_t_max * P.H);
+        it.n_sel = P.S > 1 ? P.n_sel[it.b] : kept_shared;
+        it.n_q = (it.n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
+        return it;
+    };
+    // zero rows of dq, dk, dv for every dropped variate, spread over the 16 phase warps of the whole grid; each CTA runs it once
+    bool zeros_written = P.inv_idx == nullptr;
+    auto write_zero_rows = [&]() {
+        zeros_written = true;
+        const int chunks_row = P.H * (P.D / 8);
+        const int total_rows = P.B * P.N;
+        const int lane = threadIdx.x & 31;
+        const int warps_cta = 2 * kPipeGroup / 32;
+        const int warps_grid = gridDim.x * warps_cta;
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
+        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
+        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
+        int group = 1;
+        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
+        for (int base = (blockIdx.x * warps_cta + (warp - 4)) * group; base < total_rows; base += warps_grid * group) {
+            const int r = base + lane;
+            bool dropped = false;
+            if (lane < group && r < total_rows) {
+                const int b = r / P.N, n = r - b * P.N;
+                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
+            }
+            unsigned mask = __ballot_sync(0xffffffffu, dropped);
+            while (mask) {
+                const int l = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
+                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
+            }
+        }
+    };
+    // bf16 staging of a 64-column accumulator (this thread's 32 columns of its key row), then whole 128-byte rows to the
+    // full-layout gradient: used by phase A for dV and by phase B for dK (and dQ of a single-tile instance)
+    auto stage_acc = [&](unsigned char* tile, uint32_t tm, float mul, int row, int half) {
+        float acc[32];
+        tmem_ld32(tm + lane_sel + half * 32, acc);
+        tmem_ld_wait();
+        unsigned char* rowp = tile + row * kRowBytes;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(rowp + (((half * 4 + q) ^ (row & 7)) << 4)) =
+                make_uint4(pack2(acc[8 * q + 0] * mul, acc[8 * q + 1] * mul), pack2(acc[8 * q + 2] * mul, acc[8 * q + 3] * mul),
+                           pack2(acc[8 * q + 4] * mul, acc[8 * q + 5] * mul), pack2(acc[8 * q + 6] * mul, acc[8 * q + 7] * mul));
+    };
+    auto store_rows = [&](const unsigned char* tile, __nv_bfloat16* dst, const int* nout, int gt, int b, int h) {     // gt: thread index in its group
+        const int c = gt & 7;
+        if (c * 8 >= P.D) return;
+        for (int r = gt >> 3; r < kTile; r += kPipeGroup / 8) {
+            const int n = nout[r];
+            if (n < 0) continue;
+            *reinterpret_cast<uint4*>(dst + ((static_cast<size_t>(b) * P.N + n) * P.H + h) * P.D + c * 8) =
+                *reinterpret_cast<const uint4*>(tile + r * kRowBytes + ((c ^ (r & 7)) << 4));
+        }
+    };
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ issue and dQ drain --------------------------------
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPipeSmallRegs));
+        constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);     // K-major x K-major, N = 128
+        constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major (tensor memory), B MN-major, N = 64
+        constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
+        const uint64_t d_k = umma_desc_sw128(smem_u32(sK), 16, 1024), m_k = umma_desc_sw128(smem_u32(sK), kTileBytes, 1024);
+        const uint64_t d_v = umma_desc_advance(d_k, kTileBytes);
+        const uint64_t d_q0 = umma_desc_advance(d_k, 2 * kTileBytes), d_do0 = umma_desc_advance(d_k, (2 + kQStages) * kTileBytes);
+        const uint64_t m_q0 = umma_desc_advance(m_k, 2 * kTileBytes), m_do0 = umma_desc_advance(m_k, (2 + kQStages) * kTileBytes);
+        const uint64_t m_dst = umma_desc_advance(m_k, (2 + 2 * kQStages) * kTileBytes);
+        auto issue_st = [&](uint32_t stage) {
+            const uint64_t dq_ = umma_desc_advance(d_q0, stage * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kDP / 16; ++ks)
+                tc_mma_bf16_w(tm_st, umma_desc_advance(d_k, ks * 32), umma_desc_advance(dq_, ks * 32), idesc_kk, ks > 0);
+            tc_commit_w(bar_s);
+        };
+        auto issue_dpt = [&](uint32_t stage) {
+            const uint64_t dd_ = umma_desc_advance(d_do0, stage * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kDP / 16; ++ks)
+                tc_mma_bf16_w(tm_dpt, umma_desc_advance(d_v, ks * 32), umma_desc_advance(dd_, ks * 32), idesc_kk, ks > 0);
+            tc_commit_w(bar_dp);
+        };
+        auto issue_dv = [&](uint32_t stage, uint32_t acc_on) {           // reduction over the 128 queries; P^T from tensor memory
+            const uint64_t mdo = umma_desc_advance(m_do0, stage * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks)
+                tc_mma_bf16_ta_w(tm_dv, tm_pt + ks * 8, umma_desc_advance(mdo, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
+            tc_commit_w(bar_pfree);
+        };
+        auto issue_dk = [&](uint32_t stage, uint32_t acc_on) {           // dS^T from tensor memory: queries 0..63 at column 0, 64..127 at column 64
+            const uint64_t mq = umma_desc_advance(m_q0, stage * kTileBytes);
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks)
+                tc_mma_bf16_ta_w(tm_dk, tm_dpt + (ks >> 2) * 64 + (ks & 3) * 8, umma_desc_advance(mq, ks * 2048), idesc_kmn, ks > 0 ? 1u : acc_on);
+        };
+        auto issue_dq = [&]() {                                           // reduction over the 128 keys; dS from shared memory, transposed view
+#pragma unroll
+            for (int ks = 0; ks < kTile / 16; ++ks)
+                tc_mma_bf16_w(tm_dq, umma_desc_advance(m_dst, ks * 2048), umma_desc_advance(m_k, ks * 2048), idesc_mnmn, ks > 0);
+            tc_commit_w(bar_g);
+        };
+        uint32_t n_drained = 0;                          // dQ tiles handed to phase A for draining so far
+        // Three warps issue, each its own chain of products, so that no chain waits behind another's operands (every lane runs the
+        // code, an elected lane executes each product; within a warp products complete in issue order):
+        //   warp 0   S^T and dV: the chain through P^T          warp 1   dK and dP^T: the chain through dS^T in tensor memory
+        //   warp 2   dQ: the chain through dS^T in shared memory and the drained dQ tile
+        // bar_acc collects one commit from each at the end of an item.
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const Item it = decode(item);
+            if (it.jt >= it.n_q) continue;
+            const bool single_tile = it.n_q == 1;
+            const uint32_t st0 = q_count % kQStages;
+            if (warp < 3) {
+                ok &= warp_wait(bar_kv, n_done & 1);
+                if (warp < 2) ok &= warp_wait(bar_qdo + st0, (q_count / kQStages) & 1);
+                tc_fence_after();
+                if (warp == 0) issue_st(st0);
+                else if (warp == 1) issue_dpt(st0);
+            }
+            for (int i = 0; i < it.n_q; ++i) {
+                const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
+                if (warp == 0) {
+                    ok &= warp_wait(bar_sfree, ph);      // phase A holds S^T of this tile: the next one may overwrite it
+                    if (i + 1 < it.n_q) {
+                        ok &= warp_wait(bar_qdo + st1, ((qc + 1) / kQStages) & 1);
+                        tc_fence_after();
+                        issue_st(st1);
+                    }
+                    ok &= warp_wait(bar_p, ph);
+                    tc_fence_after();
+                    issue_dv(st, i > 0);
+                } else if (warp == 1) {
+                    ok &= warp_wait(bar_ds, ph);
+                    tc_fence_after();
+                    issue_dk(st, i > 0);
+                    if (i + 1 < it.n_q) {                // over dS^T in tensor memory, behind dK which reads it
+                        ok &= warp_wait(bar_qdo + st1, ((qc + 1) / kQStages) & 1);
+                        tc_fence_after();
+                        issue_dpt(st1);
+                    }
+                } else if (warp == 2) {
+                    ok &= warp_wait(bar_ds, ph);
+                    if (n_drained > 0) ok &= warp_wait(bar_dqfree, (n_drained - 1) & 1);      // phase A has taken the previous dQ out of tensor memory
+                    tc_fence_after();
+                    issue_dq();
+                    if (!single_tile) ++n_drained;
+                }
+            }
+            if (warp < 3) tc_commit_w(bar_acc);          // this warp's products of the item
+            if (!ok) break;
+            q_count += it.n_q;
+            ++n_done;
+        }
+    } else if (warp < 12) {
+        // ------------------------------------------------------------ phase A: P^T --------------------------------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPipeBigRegs));
+        const int gt = tid - 128, row = gt & (kTile - 1), half = gt >> 7;
+        const bool owner = gt == 0;                      // the one thread that owns the bulk reductions of dQ
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const Item it = decode(item);
+            if (it.jt >= it.n_q) continue;
+            const int n_sel = it.n_sel;
+            const bool key_valid = it.jt * kTile + row < n_sel;
+            const bool single_tile = it.n_q == 1;
+            // dQ of query tile i out of tensor memory (this thread's 32 head dimensions of query row `row`) into the fp32 staging tile,
+            // which one thread adds to the accumulator with two bulk reductions; called behind a group barrier that follows the
+            // owner's wait for the previous reduction
+            auto drain = [&](int i) {
+                tc_fence_after();
+                float dqv[32];
+                tmem_ld32(tm_dq + lane_sel + half * 32, dqv);
+                tmem_ld_wait();
+                unsigned char* rowp = sDQ + half * kTileBytes + row * kRowBytes;
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    *reinterpret_cast<float4*>(rowp + ((x ^ (row & 7)) << 4)) = make_float4(dqv[4 * x], dqv[4 * x + 1], dqv[4 * x + 2], dqv[4 * x + 3]);
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(bar_dqfree);                 // the next dQ may be produced
+                ok = group_sync_and<1>(ok);              // the staging tile is complete
+                if (owner) {
+                    tma_reduce_add_4d(&map_acc, sDQ, 0, it.h, i * kTile, it.b);
+                    tma_reduce_add_4d(&map_acc, sDQ + kTileBytes, 32, it.h, i * kTile, it.b);
+                    bulk_commit_group();
+                }
+            };
+            auto load_lse = [&](int qrow) -> float {     // minus the lse of query `qrow` in the log2 domain; -inf switches a missing query off
+                return qrow < n_sel ? P.lse[(static_cast<size_t>(it.b) * P.H + it.h) * P.N + qrow] * -1.4426950408889634f : -INFINITY;
+            };
+            const uint32_t st0 = q_count % kQStages;
+            if (half == 0) {
+                s_stat[st0 * kTile + row] = load_lse(row);
+                if (it.n_q > 1) s_stat[((st0 + 1) % kQStages) * kTile + row] = load_lse(kTile + row);
+            }
+            if (!zeros_written) write_zero_rows();
+            ok = group_sync_and<1>(ok);                  // row statistics of the first tiles visible
+            for (int i = 0; i < it.n_q; ++i, ++q_count) {
+                const uint32_t st = q_count % kQStages, ph = q_count & 1, st2 = (q_count + 2) % kQStages;
+                float lse_ahead = 0.f;
+                if (i + 2 < it.n_q && half == 0) lse_ahead = load_lse((i + 2) * kTile + row);       // lands while this tile is processed
+                ok &= warp_wait_relaxed(bar_s, ph);
+                tc_fence_after();
+                float sv[64];
+                tmem_ld32(tm_st + lane_sel + half * 64, sv);
+                tmem_ld32(tm_st + lane_sel + half * 64 + 32, sv + 32);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(bar_sfree);                  // S^T is in registers
+                uint32_t pw[32];
+                {
+                    const float* lse2 = s_stat + st * kTile + half * 64;
+                    const uint64_t scale2 = pair_of(P.scale_log2, P.scale_log2);
+#pragma unroll
+                    for (int x = 0; x < 64; x += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + x);       // minus lse
+                        float e0, e1, e2, e3;
+                        halves_of(fma_pair(pair_of(sv[x + 0], sv[x + 1]), scale2, pair_of(l4.x, l4.y)), e0, e1);
+                        halves_of(fma_pair(pair_of(sv[x + 2], sv[x + 3]), scale2, pair_of(l4.z, l4.w)), e2, e3);
+                        pw[(x >> 1) + 0] = pack2(fast_exp2(e0), fast_exp2(e1));
+                        pw[(x >> 1) + 1] = pack2(fast_exp2(e2), fast_exp2(e3));
+                    }
+                    if (!key_valid) {                    // rows past n_sel hold zero keys: they must not count
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) pw[x] = 0u;
+                    }
+                }
+                if (q_count > 0) ok &= warp_wait_relaxed(bar_pfree, (q_count - 1) & 1);     // the previous P^T has been read by phase B and by dV
+                tc_fence_after();
+                tmem_st16(tm_pt + lane_sel + half * 32, pw);
+                tmem_st16(tm_pt + lane_sel + half * 32 + 16, pw + 16);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_p);                      // dV may go, phase B may read P^T
+                // dQ of the previous query tile: it was issued when phase B finished that tile
+                if (!single_tile && i > 0) {
+                    ok &= warp_wait_relaxed(bar_g, (q_count - 1) & 1);
+                    if (owner) bulk_wait_group_read0();  // the previous reduction has read the shared-memory tile
+                }
+                ok = group_sync_and<1>(ok);              // everyone is done with this tile's statistics (and agrees on ok)
+                if (!ok) break;
+                if (i + 2 < it.n_q && half == 0) s_stat[st2 * kTile + row] = lse_ahead;       // read two tiles from now, behind this barrier's successor
+                if (!single_tile && i > 0) drain(i - 1);
+            }
+            if (!ok) break;
+            if (!single_tile) {                          // dQ of the last query tile
+                ok &= warp_wait_relaxed(bar_g, (q_count - 1) & 1);
+                if (owner) bulk_wait_group_read0();
+                ok = group_sync_and<1>(ok);
+                if (!ok) break;
+                drain(it.n_q - 1);
+            }
+            // dV of this key tile
+            ok &= warp_wait_relaxed(bar_acc, n_done & 1);
+            tc_fence_after();
+            stage_acc(sdSt, tm_dv, 1.f, row, half);
+            if (owner) bulk_wait_group_read0();          // the fp32 staging tile is free (phase B may use it for a single-tile instance next)
+            tc_fence_before();
+            ok = group_sync_and<1>(ok);                  // the staging tile is complete
+            if (!ok) break;
+            // the scatter indices were written by phase B before its first arrival on bar_ds, which the products behind bar_acc waited for
+            store_rows(sdSt, P.dv, s_nout + (n_done & 1) * kTile, gt, it.b, it.h);
+            ++n_done;
+        }
+        if (owner) bulk_wait_group0();                   // the last dQ reductions have landed
+    } else {
+        // ------------------------------------------------------------ phase B: dS^T -------------------------------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPipeBigRegs));
+        const int gt = tid - 384, row = gt & (kTile - 1), half = gt >> 7, gwarp = gt >> 5;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const Item it = decode(item);
+            if (it.jt >= it.n_q) continue;
+            const int n_sel = it.n_sel, srow = P.S > 1 ? it.b : 0;
+            const bool single_tile = it.n_q == 1;
+            const int32_t* sel = P.sel_idx ? P.sel_idx + static_cast<size_t>(srow) * P.N : nullptr;
+            TileSource src = P.src, src_do = P.src_do;
+            if (src.idx) src.idx += static_cast<size_t>(srow) * P.N;
+            auto fetch_qdo = [&](int i, uint32_t stage) {    // warps 2 and 3 of the group fetch Q and dO of query tile i
+                if (gwarp == 2) {
+                    if ((tid & 31) == 0) mbar_expect_tx(bar_qdo + stage, 2 * kTileBytes);
+                    load_tile(sQ + stage * kTileBytes, &map_q, bar_qdo + stage, src, i * kTile, n_sel, it.h, it.b, P.H);
+                } else if (gwarp == 3) {
+                    load_tile(sdO + stage * kTileBytes, &map_do, bar_qdo + stage, src_do, i * kTile, n_sel, it.h, it.b, P.H);
+                }
+            };
+            auto load_delta = [&](int qrow) -> float {
+                return qrow < n_sel ? P.delta[(static_cast<size_t>(it.b) * P.H + it.h) * P.Ncap + qrow] : 0.f;
+            };
+            const int key = it.jt * kTile + row;
+            const bool key_valid = key < n_sel;
+            const uint32_t st0 = q_count % kQStages;
+            float dl_next = 0.f;
+            const float dl_first = half == 1 ? load_delta(row) : 0.f;
+            const int n_out = key_valid ? (sel ? sel[key] : key) : -1;
+            {   // every MMA of the previous item has completed: K, V and every Q/dO stage are free
+                if (gt == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
+                if (gwarp == 0) load_tile(sK, &map_k, bar_kv, src, it.jt * kTile, n_sel, it.h, it.b, P.H);
+                else if (gwarp == 1) load_tile(sV, &map_v, bar_kv, src, it.jt * kTile, n_sel, it.h, it.b, P.H);
+                fetch_qdo(0, st0);
+                if (it.n_q > 1) fetch_qdo(1, (st0 + 1) % kQStages);
+            }
+            if (half == 1) s_delta[(q_count & 1) * kTile + row] = dl_first;
+            else s_nout[(n_done & 1) * kTile + row] = n_out;     // phase A reads it at the end of the item; the array of two items ago is free
+            if (!zeros_written) write_zero_rows();
+            ok = group_sync_and<3>(ok);
+            for (int i = 0; i < it.n_q; ++i, ++q_count) {
+                const uint32_t ph = q_count & 1, st2 = (q_count + 2) % kQStages;
+                if (i + 1 < it.n_q && half == 1) dl_next = load_delta((i + 1) * kTile + row);
+                ok &= warp_wait_relaxed(bar_p, ph);
+                tc_fence_after();
+                uint32_t pw[32];                         // this thread's 64 probabilities, bf16 pairs
+                tmem_ld32(tm_pt + lane_sel + half * 32, reinterpret_cast<float*>(pw));
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(bar_pfree);
+                ok &= warp_wait_relaxed(bar_dp, ph);             // dP^T done => dK, dP^T of the previous tile are done; its S^T, dV were done when
+                                                         // P^T of this tile could be written: the ring stage of the previous tile is free
+                if (q_count > 0) ok &= warp_wait_relaxed(bar_g, (q_count - 1) & 1);      // dQ of the previous tile has read the dS^T tile in shared memory
+                tc_fence_after();
+                if (i + 2 < it.n_q) fetch_qdo(i + 2, st2);
+                {
+                    const float* dlt = s_delta + (q_count & 1) * kTile + half * 64;
+                    const uint64_t minus1 = pair_of(-1.f, -1.f);
+                    float dp[2][16];
+                    uint32_t dsw[16];
+                    // destination of this thread's key row in the two 64-query panels of the dS^T tile (128-byte swizzled rows)
+                    unsigned char* srow = sdSt + half * kTileBytes + row * kRowBytes;
+                    const int sw = row & 7;
+                    tmem_ld16(tm_dpt + lane_sel + half * 64, dp[0]);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        tmem_ld_wait();
+                        if (c < 3) tmem_ld16(tm_dpt + lane_sel + half * 64 + (c + 1) * 16, dp[(c + 1) & 1]);
+                        const float* d = dp[c & 1];
+                        uint32_t* out = dsw + (c & 1) * 8;
+#pragma unroll
+                        for (int x = 0; x < 16; x += 4) {
+                            const float4 da = *reinterpret_cast<const float4*>(dlt + c * 16 + x);
+                            const uint32_t w0 = pw[c * 8 + (x >> 1)], w1 = pw[c * 8 + (x >> 1) + 1];
+                            const uint64_t p01 = pair_of(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xFFFF0000u));
+                            const uint64_t p23 = pair_of(__uint_as_float(w1 << 16), __uint_as_float(w1 & 0xFFFF0000u));
+                            float r0, r1, r2, r3;
+                            halves_of(mul_pair(p01, fma_pair(pair_of(da.x, da.y), minus1, pair_of(d[x + 0], d[x + 1]))), r0, r1);
+                            halves_of(mul_pair(p23, fma_pair(pair_of(da.z, da.w), minus1, pair_of(d[x + 2], d[x + 3]))), r2, r3);
+                            out[(x >> 1) + 0] = pack2(r0, r1);        // rounded once: the same words go to shared and to tensor memory
+                            out[(x >> 1) + 1] = pack2(r2, r3);
+                        }
+                        *reinterpret_cast<uint4*>(srow + (((2 * c) ^ sw) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+                        *reinterpret_cast<uint4*>(srow + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+                        if (c & 1) tmem_st16(tm_dpt + lane_sel + half * 64 + (c >> 1) * 16, dsw);      // over columns this thread has consumed
+                    }
+                }
+                if (i + 1 < it.n_q && half == 1) s_delta[((q_count + 1) & 1) * kTile + row] = dl_next;
+                tmem_st_wait();
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(bar_ds);                     // dQ, dK and the next dP^T may go
+                ok = group_sync_and<3>(ok);
+                if (!ok) break;
+            }
+            if (!ok) break;
+            ok &= warp_wait_relaxed(bar_acc, n_done & 1);
+            tc_fence_after();
+            stage_acc(sdSt + kTileBytes, tm_dk, P.scale, row, half);
+            if (single_tile) stage_acc(sDQ, tm_dq, P.scale, row, half);         // complete: bar_acc covers every product of the item
+            tc_fence_before();
+            ok = group_sync_and<3>(ok);
+            if (!ok) break;
+            store_rows(sdSt + kTileBytes, P.dk, s_nout + (n_done & 1) * kTile, gt, it.b, it.h);
+            if (single_tile) store_rows(sDQ, P.dq, s_nout + (n_done & 1) * kTile, gt, it.b, it.h);
+            ++n_done;
+        }
+    }
+    if (!zeros_written && warp >= 4) write_zero_rows();          // every item of this CTA was skipped (short instances)
+    if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kBwdTmemCols);
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // dq from the accumulator (paths with many key tiles)
 // ---------------------------------------------------------------------------------------------------------
 struct ConvertParams {
@@ -793,13 +1304,19 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
     cudaGetDevice(&dev);
     if (attr_dev != dev) {
         if (int st = check_cuda(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmemBytes), "attention: smem attribute")) return st;
+        if (int st = check_cuda(cudaFuncSetAttribute(attn_bwd_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmemBytes), "attention: smem attribute")) return st;
         attr_dev = dev;
     }
+    // Many query tiles per key tile: the kernel with one warpgroup pair per phase (it needs the precomputed Delta and boxed tiles,
+    // which is what these shapes have).  The kept count is only known on the device, so the host goes by the largest it can be.
+    const bool pipelined = !gathered && pre_delta && (sel_idx ? c.N > 2048 : c.N > 2 * kTile);
     {
         const long long worst = static_cast<long long>(w.Ncap / kTile) * c.H * c.B;
         const int grid = static_cast<int>(worst < sm_count() ? worst : sm_count());      // one CTA per SM (all of tensor memory)
         LaunchScope ls_(K_ATTN_BWD, stream);
-        const cudaError_t err = launch_chained(attn_bwd_kernel, dim3(grid), dim3(kBwdThreads), kBwdSmemBytes, stream, mq, mk, mv, mdo, macc, P);
+        const cudaError_t err = pipelined
+            ? launch_chained(attn_bwd_pipe_kernel, dim3(grid), dim3(kPipeThreads), kPipeSmemBytes, stream, mq, mk, mv, mdo, macc, P)
+            : launch_chained(attn_bwd_kernel, dim3(grid), dim3(kBwdThreads), kBwdSmemBytes, stream, mq, mk, mv, mdo, macc, P);
         if (int st = check_cuda(err, "attention: backward launch")) return st;
     }
     if (!gathered && c.N > kTile) {         // several key tiles possible: dq comes from the accumulator in a pass of its own
