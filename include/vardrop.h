@@ -206,8 +206,12 @@ int vardrop_gather_rows(const float* x, const int32_t* sel_idx, const int32_t* n
  *   lse_i = log sum_j exp(S_ij).
  * bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before the second product.
  *
- * cfg (host)  B, N, H, D (D = 32 or 64; N <= 65536), sm_scale (0 selects 1/sqrt(D)), S (1 or B).
- * q, k, v     [B, N, H, D] bf16, contiguous.
+ * cfg (host)  B, N, H, D (D = 32 or 64; N <= 65536), sm_scale (0 selects 1/sqrt(D)), S (1 or B), and the element strides
+ *             sB, sN, sH of q, k and v (the head dimension is contiguous): element (b, n, h, d) of each lies at
+ *             b sB + n sN + h sH + d.  All three 0 selects the contiguous layout sH = D, sN = H D, sB = N H D; otherwise
+ *             each must be a multiple of 8 elements (16 bytes), sH >= D, sN >= sH, sB >= sN (views of a fused [B, N, 3, H, D]
+ *             projection, padded heads or tokens, slices along N).  o, lse, d_o, dq, dk, dv are always contiguous.
+ * q, k, v     [B, N, H, D] bf16 with the strides above.
  * sel_idx     [S, N] int32, ascending kept variates (vardrop_select's output: S = 1 for the paper's batch-wise
  *             grouping, S = B when every instance was hashed and sampled on its own), or NULL for the
  *             all-token path (VarDrop off, the inference / "ground" configuration of the paper).
@@ -222,6 +226,7 @@ typedef struct {
     int32_t B, N, H, D;
     float sm_scale;
     int32_t S;      /* selections: 0 or 1 = one shared by all instances (batch-wise grouping), B = one per instance */
+    int64_t sB, sN, sH;   /* element strides of q, k, v; all 0 = contiguous */
 } vardrop_attn_cfg;
 
 size_t vardrop_attn_workspace_bytes(const vardrop_attn_cfg* cfg);

@@ -30,7 +30,8 @@ class SelectCfg(C.Structure):
 
 
 class AttnCfg(C.Structure):
-    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float), ("S", C.c_int32)]
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("sm_scale", C.c_float), ("S", C.c_int32),
+                ("sB", C.c_int64), ("sN", C.c_int64), ("sH", C.c_int64)]          # element strides of q, k, v; all 0 = contiguous
 
 
 class GatherCfg(C.Structure):

@@ -1239,8 +1239,10 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
                     const int32_t* sel_idx, const int32_t* n_sel, const int32_t* inv_idx, const vardrop_attn_cfg& c, void* dq,
                     void* dk, void* dv, void* ws, cudaStream_t stream) {
     const AttnWs w = attn_layout(c);
+    const QkvLayout L = qkv_layout(c);
     char* base = static_cast<char*>(ws);
     const bool staged = attn_uses_staging(c, sel_idx);
+    const long long Hd = static_cast<long long>(c.H) * kDP, HD = static_cast<long long>(c.H) * c.D;
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
 
     const bool gathered = attn_uses_gather(c, sel_idx);
@@ -1267,30 +1269,31 @@ int attn_bwd_launch(const void* q, const void* k, const void* v, const void* o, 
 
     CUtensorMap mq, mk, mv, mdo;
     if (staged) {
-        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
-        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
-        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
-        if (int st = make_tile_map(&mdo, base + w.dog, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
+        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
+        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
+        if (int st = make_tile_map(&mdo, base + w.dog, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
     } else if (gathered) {
-        const long long rows = static_cast<long long>(c.B) * c.N * c.H;
-        if (int st = make_row_map(&mq, q, rows)) return st;
-        if (int st = make_row_map(&mk, k, rows)) return st;
-        if (int st = make_row_map(&mv, v, rows)) return st;
-        if (int st = make_row_map(&mdo, d_o, rows)) return st;
+        if (int st = make_row_map(&mq, q, L.rows_total, L.sH)) return st;
+        if (int st = make_row_map(&mk, k, L.rows_total, L.sH)) return st;
+        if (int st = make_row_map(&mv, v, L.rows_total, L.sH)) return st;
+        if (int st = make_row_map(&mdo, d_o, static_cast<long long>(c.B) * c.N * c.H, kDP)) return st;      // d_o is contiguous
     } else {
-        if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
-        if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
-        if (int st = make_tile_map(&mv, v, c.B, c.N, c.N, c.H)) return st;
-        if (int st = make_tile_map(&mdo, d_o, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mq, q, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
+        if (int st = make_tile_map(&mk, k, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
+        if (int st = make_tile_map(&mv, v, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
+        if (int st = make_tile_map(&mdo, d_o, c.B, c.N, c.H, c.N * HD, HD, c.D)) return st;
     }
     CUtensorMap macc;
     if (int st = make_acc_map(&macc, base + w.dq_acc, c.B, w.Ncap, c.H)) return st;
     BwdParams P{};
     P.lse = lse; P.o = static_cast<const __nv_bfloat16*>(o); P.delta = pre_delta ? reinterpret_cast<const float*>(base + w.delta) : nullptr;
     P.dq_acc = reinterpret_cast<float*>(base + w.dq_acc);
-    P.src.idx = sel_idx; P.src.gathered = gathered ? 1 : 0; P.src.tokens = c.N; P.src.rows_total = c.B * c.N * c.H;
+    P.src.idx = sel_idx; P.src.gathered = gathered ? 1 : 0; P.src.tokens = c.N;
+    P.src.rows_total = static_cast<int>(L.rows_total); P.src.row_b = static_cast<int>(L.row_b); P.src.row_n = static_cast<int>(L.row_n);
     P.src_do = P.src;
-    P.src_do.idx = nullptr;         // dO rows are already compact: slot j is row j
+    P.src_do.idx = nullptr;         // dO rows are already compact: slot j is row j (and d_o is contiguous)
+    P.src_do.rows_total = c.B * c.N * c.H; P.src_do.row_b = c.N * c.H; P.src_do.row_n = c.H;
     P.dq = static_cast<__nv_bfloat16*>(dq); P.dk = static_cast<__nv_bfloat16*>(dk); P.dv = static_cast<__nv_bfloat16*>(dv);
     P.sel_idx = sel_idx; P.n_sel = sel_idx ? n_sel : nullptr;
     P.inv_idx = sel_idx ? inv_idx : nullptr;

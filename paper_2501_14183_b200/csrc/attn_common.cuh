@@ -43,7 +43,7 @@ inline AttnWs attn_layout(const vardrop_attn_cfg& c) {
 // `token_stride` the allocated tokens per instance.
 // Tensor map over the same memory seen as [rows, 64] bf16 (rows = B * tokens * H) for row gathers: box = one row,
 // 128-byte swizzle, rows outside the tensor read as zero.
-int make_row_map(CUtensorMap* map, const void* base, long long rows);
+int make_row_map(CUtensorMap* map, const void* base, long long rows, long long row_stride_elems);
 
 // Tensor map over the fp32 dQ' accumulator [B, Ncap, H, 64]: box = 128 tokens x 32 floats (one 128-byte swizzled row
 // per token) of one head, the unit of the backward kernel's bulk reduce-add.
@@ -52,7 +52,28 @@ int make_acc_map(CUtensorMap* map, const void* base, int B, int Ncap, int H);
 // Number of SMs of the current device (cached per thread and device).
 int sm_count();
 
-int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int token_stride, int H);
+int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int H, long long sB, long long sN, long long sH);
+
+// Element strides of q, k, v as the kernels see them.  The row view (one 64-element row per (instance, token, head), rows a
+// constant distance apart) exists when sN and sB are multiples of sH: row(b, n, h) = b row_b + n row_n + h.
+struct QkvLayout {
+    long long sB, sN, sH;       // element strides
+    bool row_linear;            // the row view exists
+    long long rows_total;       // rows of that view (one past the last is the zero row of the gathers)
+    long long row_b, row_n;
+};
+inline QkvLayout qkv_layout(const vardrop_attn_cfg& c) {
+    QkvLayout L;
+    const bool dflt = c.sB == 0 && c.sN == 0 && c.sH == 0;
+    L.sH = dflt ? c.D : c.sH;
+    L.sN = dflt ? static_cast<long long>(c.H) * c.D : c.sN;
+    L.sB = dflt ? static_cast<long long>(c.N) * c.H * c.D : c.sB;
+    L.row_linear = L.sN % L.sH == 0 && L.sB % L.sH == 0;
+    L.row_n = L.row_linear ? L.sN / L.sH : 0;
+    L.row_b = L.row_linear ? L.sB / L.sH : 0;
+    L.rows_total = L.row_linear ? (c.B - 1) * L.row_b + (c.N - 1) * L.row_n + c.H : 0;
+    return L;
+}
 
 // First 1024-byte boundary at or after p (swizzled tiles need it).
 __device__ __forceinline__ unsigned char* align_tiles(unsigned char* p) {
@@ -68,7 +89,8 @@ struct TileSource {
     const int32_t* idx;    // gather indices of the instance's selection (NULL: identity)
     int gathered;          // 0: tiled box, 1: row gathers
     int tokens;            // tokens per instance in the gathered tensor
-    int rows_total;        // B * tokens * H
+    int rows_total;        // rows of the [rows, 64] view; row(b, n, h) = b row_b + n row_n + h
+    int row_b, row_n;
 };
 // Rows of the [rows, 64] view that the four slots tok0 + 4 lane .. + 3 of a gathered tile name (a row past the end for
 // slots at or past n_valid).  `picks` are the four entries idx[tok0 + 4 lane ..] (see tile_picks), fetched ahead of
@@ -95,7 +117,7 @@ __device__ __forceinline__ void load_tile_picked(unsigned char* dst, const CUten
     const int n[4] = {picks.x, picks.y, picks.z, picks.w};
     int rows[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) rows[e] = (slot + e < n_valid && n[e] >= 0) ? (b * src.tokens + n[e]) * H + h : src.rows_total;
+    for (int e = 0; e < 4; ++e) rows[e] = (slot + e < n_valid && n[e] >= 0) ? b * src.row_b + n[e] * src.row_n + h : src.rows_total;
     tma_gather4(dst + lane * 4 * kRowBytes, map, bar, 0, rows[0], rows[1], rows[2], rows[3]);
 }
 __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* map, uint64_t* bar, const TileSource& src, int tok0, int n_valid,
@@ -126,7 +148,11 @@ __device__ __forceinline__ int max_kept(const int32_t* n_sel, int S, int N, int*
     return *scratch;
 }
 
-inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D != kDP || (sel_idx != nullptr && c.N > kGatherMaxN); }
-inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D == kDP && sel_idx != nullptr && c.N <= kGatherMaxN; }
+// (row gathers also need the row view of the caller's strides and row indices that fit 31 bits; other layouts are staged)
+inline bool attn_uses_gather(const vardrop_attn_cfg& c, const int32_t* sel_idx) {
+    const QkvLayout L = qkv_layout(c);
+    return c.D == kDP && sel_idx != nullptr && c.N <= kGatherMaxN && L.row_linear && L.rows_total < (1ll << 31);
+}
+inline bool attn_uses_staging(const vardrop_attn_cfg& c, const int32_t* sel_idx) { return c.D != kDP || (sel_idx != nullptr && !attn_uses_gather(c, sel_idx)); }
 
 }  // namespace vardrop

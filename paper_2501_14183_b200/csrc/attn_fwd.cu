@@ -42,6 +42,7 @@ struct MapKey {
 struct alignas(64) MapSlot {
     CUtensorMap map;
     MapKey key;
+    long long aux[3];      // strides of a tile map (the key only carries a mix of them)
     bool used;
 };
 constexpr int kMapSlots = 256;
@@ -63,16 +64,15 @@ int sm_count() {
     return cached;
 }
 
-int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int token_stride, int H) {
-    const MapKey key{base, 0, 1, B, tokens, token_stride * 65536 + H};
+int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int H, long long sB, long long sN, long long sH) {
+    const MapKey key{base, sB * 131 + sN * 31 + sH, 1, B, tokens, H};
     MapSlot* slot = map_slot(key);
-    if (slot->used && slot->key == key) { *map = slot->map; return VARDROP_OK; }
+    if (slot->used && slot->key == key && slot->aux[0] == sB && slot->aux[1] == sN && slot->aux[2] == sH) { *map = slot->map; return VARDROP_OK; }
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(kDP), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(tokens),
                                 static_cast<cuuint64_t>(B)};
-    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kRowBytes), static_cast<cuuint64_t>(H) * kRowBytes,
-                                   static_cast<cuuint64_t>(token_stride) * H * kRowBytes};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(sH) * 2, static_cast<cuuint64_t>(sN) * 2, static_cast<cuuint64_t>(sB) * 2};
     const cuuint32_t box[4] = {kDP, 1, kTile, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -80,17 +80,18 @@ int make_tile_map(CUtensorMap* map, const void* base, int B, int tokens, int tok
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r));
     slot->map = *map; slot->key = key; slot->used = true;
+    slot->aux[0] = sB; slot->aux[1] = sN; slot->aux[2] = sH;
     return VARDROP_OK;
 }
 
-int make_row_map(CUtensorMap* map, const void* base, long long rows) {
-    const MapKey key{base, rows, 2, 0, 0, 0};
+int make_row_map(CUtensorMap* map, const void* base, long long rows, long long row_stride_elems) {
+    const MapKey key{base, rows, 2, static_cast<int>(row_stride_elems), 0, 0};
     MapSlot* slot = map_slot(key);
     if (slot->used && slot->key == key) { *map = slot->map; return VARDROP_OK; }
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(VARDROP_ERR_CUDA, "attention: cuTensorMapEncodeTiled entry point not available");
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(kDP), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(kRowBytes)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(row_stride_elems) * 2};
     const cuuint32_t box[2] = {kDP, 1};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -126,6 +127,12 @@ int attn_validate(const vardrop_attn_cfg& c) {
     if (c.H > 65535 || c.B > 65535) return fail(VARDROP_ERR_UNSUPPORTED, "attention: B or H above 65535");
     if (c.S != 0 && c.S != 1 && c.S != c.B) return fail(VARDROP_ERR_INVALID_ARG, "attention: S=%d must be 1 (shared selection) or B (one per instance)", c.S);
     if (!(c.sm_scale >= 0.f)) return fail(VARDROP_ERR_INVALID_ARG, "attention: sm_scale must be >= 0 (0 selects 1/sqrt(D))");
+    if (c.sB != 0 || c.sN != 0 || c.sH != 0) {
+        if (c.sH < c.D || c.sN < c.sH || c.sB < c.sN || (c.sH | c.sN | c.sB) % 8 != 0)
+            return fail(VARDROP_ERR_INVALID_ARG, "attention: strides sB=%lld sN=%lld sH=%lld must be multiples of 8 with sB >= sN >= sH >= D (or all 0)",
+                        static_cast<long long>(c.sB), static_cast<long long>(c.sN), static_cast<long long>(c.sH));
+        if (c.sB > (1ll << 38)) return fail(VARDROP_ERR_UNSUPPORTED, "attention: sB above 2^38 elements");
+    }
     return VARDROP_OK;
 }
 
@@ -142,6 +149,7 @@ struct GatherParams {
     const int32_t* sel_idx;   // NULL: identity
     const int32_t* n_sel;     // NULL with sel_idx NULL
     int N, Ncap, H, D, S;     // S selection rows (1: shared, B: per instance)
+    long long cB, cN, cH;     // strides of the sources in 16-byte chunks
 };
 
 __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
@@ -155,7 +163,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
     const int chunks_row = P.H * (kDP / 8);                                   // 16-byte chunks per staged token
     const int src_chunks_head = P.D / 8;
     const int total = n_fill * chunks_row;
-    const uint4* src_b = P.src[t] + static_cast<size_t>(b) * P.N * (P.H * src_chunks_head);
+    const uint4* src_b = P.src[t] + static_cast<size_t>(b) * P.cB;
     uint4* dst_b = P.dst[t] + static_cast<size_t>(b) * P.Ncap * chunks_row;
     // four chunks per thread and trip, a whole CTA apart, so that four independent row lookups and four 16-byte loads are in
     // flight per thread before the first store (one load per trip leaves the memory system idle most of the time)
@@ -173,7 +181,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams P) {
                 const int h = c / (kDP / 8), dc = c - h * (kDP / 8);
                 if (j < n_sel && dc < src_chunks_head) {
                     const int n = sel ? __ldg(sel + j) : j;
-                    from[u] = src_b + static_cast<size_t>(n) * (P.H * src_chunks_head) + h * src_chunks_head + dc;
+                    from[u] = src_b + static_cast<size_t>(n) * P.cN + static_cast<size_t>(h) * P.cH + dc;
                 }
             }
         }
@@ -854,8 +862,10 @@ static bool attn_fwd_uses_groups(const vardrop_attn_cfg& c, const int32_t* sel_i
 int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* sel_idx, const int32_t* n_sel,
                     const vardrop_attn_cfg& c, void* o, float* lse, void* ws, cudaStream_t stream) {
     const AttnWs w = attn_layout(c);
+    const QkvLayout L = qkv_layout(c);
     char* base = static_cast<char*>(ws);
     const bool staged = attn_uses_staging(c, sel_idx);
+    const long long Hd = static_cast<long long>(c.H) * kDP;          // staged copies: [B, Ncap, H, 64] contiguous
     CUtensorMap mq, mk, mv;
     if (staged) {
         GatherParams G{};
@@ -864,6 +874,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         G.dst[2] = reinterpret_cast<uint4*>(base + w.vg);
         G.sel_idx = sel_idx; G.n_sel = sel_idx ? n_sel : nullptr;
         G.N = c.N; G.Ncap = w.Ncap; G.H = c.H; G.D = c.D; G.S = attn_sel_rows(c);
+        G.cB = L.sB / 8; G.cN = L.sN / 8; G.cH = L.sH / 8;
         const long long work = static_cast<long long>(w.Ncap) * c.H * (kDP / 8);
         int gx = static_cast<int>((work + 255) / 256);
         const int cap = max(1, 8 * sm_count() / (3 * c.B));        // about eight CTAs per SM in total (the kept count is only known on the
@@ -872,18 +883,17 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
         cudaError_t gerr;
         { LaunchScope ls_(K_GATHER, stream); gerr = launch_chained(gather_kernel, dim3(gx, c.B, 3), dim3(256), 0, stream, G); }
         if (int st = check_cuda(gerr, "attention: gather launch")) return st;
-        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, w.Ncap, c.H)) return st;
-        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, w.Ncap, c.H)) return st;
-        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, w.Ncap, c.H)) return st;
+        if (int st = make_tile_map(&mq, base + w.qg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
+        if (int st = make_tile_map(&mk, base + w.kg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
+        if (int st = make_tile_map(&mv, base + w.vg, c.B, w.Ncap, c.H, w.Ncap * Hd, Hd, kDP)) return st;
     } else if (attn_uses_gather(c, sel_idx)) {
-        const long long rows = static_cast<long long>(c.B) * c.N * c.H;
-        if (int st = make_row_map(&mq, q, rows)) return st;
-        if (int st = make_row_map(&mk, k, rows)) return st;
-        if (int st = make_row_map(&mv, v, rows)) return st;
+        if (int st = make_row_map(&mq, q, L.rows_total, L.sH)) return st;
+        if (int st = make_row_map(&mk, k, L.rows_total, L.sH)) return st;
+        if (int st = make_row_map(&mv, v, L.rows_total, L.sH)) return st;
     } else {
-        if (int st = make_tile_map(&mq, q, c.B, c.N, c.N, c.H)) return st;
-        if (int st = make_tile_map(&mk, k, c.B, c.N, c.N, c.H)) return st;
-        if (int st = make_tile_map(&mv, v, c.B, c.N, c.N, c.H)) return st;
+        if (int st = make_tile_map(&mq, q, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
+        if (int st = make_tile_map(&mk, k, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
+        if (int st = make_tile_map(&mv, v, c.B, c.N, c.H, L.sB, L.sN, L.sH)) return st;
     }
     FwdParams P{};
     P.o = static_cast<__nv_bfloat16*>(o); P.lse = lse; P.n_sel = sel_idx ? n_sel : nullptr;
@@ -891,7 +901,7 @@ int attn_fwd_launch(const void* q, const void* k, const void* v, const int32_t* 
     P.dq_acc = reinterpret_cast<float4*>(base + w.dq_acc);
     P.tile_done = reinterpret_cast<int32_t*>(base + w.tile_done);
     P.src.idx = sel_idx; P.src.gathered = attn_uses_gather(c, sel_idx) ? 1 : 0; P.src.tokens = c.N;
-    P.src.rows_total = c.B * c.N * c.H;
+    P.src.rows_total = static_cast<int>(L.rows_total); P.src.row_b = static_cast<int>(L.row_b); P.src.row_n = static_cast<int>(L.row_n);
     P.B = c.B; P.N = c.N; P.Ncap = w.Ncap; P.H = c.H; P.D = c.D; P.S = attn_sel_rows(c);
     const float scale = c.sm_scale > 0.f ? c.sm_scale : 1.f / sqrtf(static_cast<float>(c.D));
     P.scale_log2 = scale * 1.4426950408889634f;

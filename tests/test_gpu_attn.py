@@ -210,3 +210,72 @@ def test_attention_per_instance_selections():
             assert_attn_close(g, want, f"{name}[{b}]")
             assert np.all(g[:, np.setdiff1d(np.arange(N), s_)] == 0.0)
         assert torch.isnan(o[b, c:].float()).all()
+
+
+def run_strided(q, k, v, d_full, B, N, H, D, sel):
+    """q, k, v are (possibly non-contiguous) views [B, N, H, D] with a contiguous head dimension; their strides go into the config."""
+    assert q.stride() == k.stride() == v.stride() and q.stride(3) == 1
+    cfg = vd.AttnCfg(B, N, H, D, 0.0, 1, q.stride(0), q.stride(1), q.stride(2))
+    ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
+    o = torch.full((B, N, H, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, H, N), float("nan"), dtype=torch.float32, device="cuda")
+    if sel is None:
+        Ns, sel_t, nsel_t, inv_t, d_o = N, None, None, None, d_full
+    else:
+        Ns = len(sel)
+        sel_pad = np.full(N, -1, np.int32); sel_pad[:Ns] = sel
+        inv = np.full(N, -1, np.int32); inv[sel] = np.arange(Ns, dtype=np.int32)
+        sel_t, inv_t = torch.from_numpy(sel_pad).cuda(), torch.from_numpy(inv).cuda()
+        nsel_t = torch.tensor([Ns], dtype=torch.int32, device="cuda")
+        d_o = torch.full((B, N, H, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        d_o[:, :Ns] = d_full[:, :Ns]
+    vd.vardrop_attn_fwd(q, k, v, sel_t, nsel_t, cfg, o, lse, ws)
+    dq, dk, dv = (torch.full((B, N, H, D), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, sel_t, nsel_t, inv_t, cfg, dq, dk, dv, ws)
+    torch.cuda.synchronize()
+    assert vd.ws_status(ws) == vd.OK
+    f = lambda t: t.double().cpu().numpy()
+    return f(o)[:, :Ns], f(lse)[:, :, :Ns], f(dq), f(dk), f(dv)
+
+
+@pytest.mark.parametrize("layout", ["fused_qkv", "padded_heads", "padded_tokens", "token_slice"])
+@pytest.mark.parametrize("B,N,H,D,Ns", [(2, 300, 2, 64, 140), (1, 700, 2, 64, 300), (2, 200, 3, 64, None), (1, 600, 2, 64, None), (2, 90, 2, 32, 50)])
+def test_attention_strided_qkv(layout, B, N, H, D, Ns):
+    """q, k, v as views of larger buffers (the element strides of the configuration): slices of a fused [B, N, 3, H, D] projection,
+    heads padded to D + 8, tokens padded by 8 elements (no row view: the library stages), and a slice along N of a longer
+    sequence.  Results must match the oracle run on contiguous copies."""
+    dev, ref = bf16_tokens(B, N, H, D, 0.5, seed=N + H)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    junk = lambda *shape: (torch.rand(shape, device="cuda", generator=gen) * 8 - 4).to(torch.bfloat16)       # what lies between the rows
+    if layout == "fused_qkv":
+        buf = junk(B, N, 3, H, D)
+        views = [buf[:, :, i] for i in range(3)]
+    elif layout == "padded_heads":
+        bufs = [junk(B, N, H, D + 8) for _ in range(3)]
+        views = [b[..., :D] for b in bufs]
+    elif layout == "padded_tokens":
+        bufs = [junk(B, N, H * D + 8) for _ in range(3)]
+        views = [b[..., : H * D].unflatten(-1, (H, D)) for b in bufs]
+    else:
+        bufs = [junk(B, N + 37, H, D) for _ in range(3)]
+        views = [b[:, 16: 16 + N] for b in bufs]
+    for view, t in zip(views, dev[:3]):
+        view.copy_(t)
+    sel = None if Ns is None else pick(N, Ns, seed=N)
+    o, lse, dq, dk, dv = run_strided(views[0], views[1], views[2], dev[3], B, N, H, D, sel)
+    n_rows = N if sel is None else len(sel)
+    wo, wl = oracle.attn_fwd(ref[0], ref[1], ref[2], sel)
+    wq, wk, wv = oracle.attn_bwd(ref[0], ref[1], ref[2], ref[3][:, :n_rows], sel)
+    for got, want, name in ((o, wo, "o"), (lse, wl, "lse"), (dq, wq, "dq"), (dk, wk, "dk"), (dv, wv, "dv")):
+        assert_attn_close(got, want, f"{layout} {name}")
+
+
+def test_attention_stride_validation():
+    q = torch.zeros((1, 8, 2, 64), dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros_like(q)
+    lse = torch.zeros((1, 2, 8), device="cuda")
+    ws = vd.alloc_ws(1 << 20)
+    for strides in [(8 * 128, 128, 60), (8 * 128, 132, 64), (100, 128, 64), (8 * 128, 64, 128)]:
+        with pytest.raises(vd.VardropError) as e:
+            vd.vardrop_attn_fwd(q, q, q, None, None, vd.AttnCfg(1, 8, 2, 64, 0.0, 1, *strides), o, lse, ws)
+        assert e.value.status == vd.ERR_INVALID_ARG

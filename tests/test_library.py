@@ -48,7 +48,7 @@ def test_status_strings_and_version(lib):
 def test_struct_layouts_match_header():
     assert C.sizeof(vd.HashCfg) == 28
     assert C.sizeof(vd.SelectCfg) == 40 and vd.SelectCfg.rate.offset == 16 and vd.SelectCfg.seed.offset == 24
-    assert C.sizeof(vd.AttnCfg) == 24
+    assert C.sizeof(vd.AttnCfg) == 48 and vd.AttnCfg.sB.offset == 24
 
 
 def test_workspace_queries_need_no_gpu(lib):
