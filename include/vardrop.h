@@ -241,7 +241,9 @@ int vardrop_attn_fwd(const void* q, const void* k, const void* v, const int32_t*
  * then scattered: row sel_idx[i] of dq/dk/dv receives row i of dQ'/dK'/dV'; rows of dropped variates
  * are written as zeros, so every row of dq, dk, dv is written exactly once.
  *
- * q, k, v, sel_idx, n_sel, cfg, ws   as given to vardrop_attn_fwd (ws unmodified since).
+ * q, k, v, sel_idx, n_sel, cfg, ws   as given to vardrop_attn_fwd (ws unmodified since).  Exactly one backward call per forward
+ *             call on a workspace: a backward call that finds no unconsumed forward pass in `ws` (called twice, or after another
+ *             forward call reused the workspace and was already consumed) sets the device status to VARDROP_ERR_INVALID_ARG.
  * o, lse      outputs of vardrop_attn_fwd.
  * d_o         [B, N, H, D] bf16, gradient of o; rows 0..n_sel-1 are read.
  * inv_idx     [S, N] int32 from vardrop_select (NULL when sel_idx is NULL).

@@ -251,6 +251,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const uint32_t tmem = *tmem_slot;
     chain_wait();
     chain_release();
+    // One backward pass per forward pass: the forward kernel cleared this workspace's dQ' accumulator and tile counters and left a
+    // mark; a backward pass that does not find the mark (a second backward for the same forward, or two forwards sharing the
+    // workspace before their backwards) would add into stale state, so it reports the call instead of returning wrong gradients.
+    if (blockIdx.x == 0 && threadIdx.x == 0 && atomicExch(P.status + kWsPairingWord, 0) != 1) set_status(P.status, VARDROP_ERR_INVALID_ARG);
     // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
     const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 100)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
@@ -796,6 +800,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
     const uint32_t tmem = *tmem_slot;
     chain_wait();
     chain_release();
+    // One backward pass per forward pass: the forward kernel cleared this workspace's dQ' accumulator and tile counters and left a
+    // mark; a backward pass that does not find the mark (a second backward for the same forward, or two forwards sharing the
+    // workspace before their backwards) would add into stale state, so it reports the call instead of returning wrong gradients.
+    if (blockIdx.x == 0 && threadIdx.x == 0 && atomicExch(P.status + kWsPairingWord, 0) != 1) set_status(P.status, VARDROP_ERR_INVALID_ARG);
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
     const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, s_scratch) : kept_shared) + kTile - 1) / kTile;
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles

@@ -334,6 +334,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
     const uint32_t tmem = *tmem_slot;
     chain_wait();
     chain_release();
+    if (blockIdx.x == 0 && threadIdx.x == 0) P.status[kWsPairingWord] = 1;      // this workspace now holds a forward pass that no backward pass has consumed
     // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
     const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, s_scratch) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
@@ -668,6 +669,7 @@ __global__ void __launch_bounds__(kTileFwdThreads) attn_fwd_tile_kernel(const __
     const uint32_t tmem = *tmem_slot;
     chain_wait();
     chain_release();
+    if (blockIdx.x == 0 && threadIdx.x == 0) P.status[kWsPairingWord] = 1;      // this workspace now holds a forward pass that no backward pass has consumed
     // kept count of a selection shared by the batch: one broadcast load (per-instance selections take the maximum)
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
     const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 48)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection

@@ -17,6 +17,7 @@ int check_cuda(cudaError_t e, const char* what);     // VARDROP_OK or VARDROP_ER
 
 // Every workspace starts with this header; word 0 is the device-side status (a vardrop_status).
 constexpr size_t kWsHeaderBytes = 256;
+constexpr int kWsPairingWord = 1;      // attention workspace: 1 while a forward pass awaits its backward pass
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -279,3 +279,26 @@ def test_attention_stride_validation():
         with pytest.raises(vd.VardropError) as e:
             vd.vardrop_attn_fwd(q, q, q, None, None, vd.AttnCfg(1, 8, 2, 64, 0.0, 1, *strides), o, lse, ws)
         assert e.value.status == vd.ERR_INVALID_ARG
+
+
+def test_backward_without_a_fresh_forward_is_reported():
+    """The forward pass leaves state for exactly one backward pass in the workspace; a second backward on it is flagged in the
+    device status word instead of silently adding into a consumed accumulator."""
+    B, N, H, D = 1, 300, 2, 64
+    dev, _ = bf16_tokens(B, N, H, D, 1.0, seed=3)
+    q, k, v, d_o = dev
+    cfg = vd.AttnCfg(B, N, H, D, 0.0)
+    ws = vd.alloc_ws(vd.vardrop_attn_workspace_bytes(cfg))
+    o = torch.zeros_like(q); lse = torch.zeros((B, H, N), device="cuda")
+    dq, dk, dv = (torch.zeros_like(q) for _ in range(3))
+    vd.vardrop_attn_fwd(q, k, v, None, None, cfg, o, lse, ws)
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, None, None, None, cfg, dq, dk, dv, ws)
+    assert vd.ws_status(ws) == vd.OK
+    first = dq.clone()
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, None, None, None, cfg, dq, dk, dv, ws)          # no forward in between
+    assert vd.ws_status(ws) == vd.ERR_INVALID_ARG
+    ws[:4] = 0                                                                                 # the caller clears the word ...
+    vd.vardrop_attn_fwd(q, k, v, None, None, cfg, o, lse, ws)                                  # ... and the pair works again
+    vd.vardrop_attn_bwd(q, k, v, o, lse, d_o, None, None, None, cfg, dq, dk, dv, ws)
+    assert vd.ws_status(ws) == vd.OK
+    np.testing.assert_allclose(dq.float().cpu().numpy(), first.float().cpu().numpy(), rtol=0, atol=2e-3)
