@@ -203,3 +203,59 @@ def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
     assert np.array_equal(keys.cpu().numpy().view(np.uint64), want)
     with pytest.raises(vd.VardropError):
         vd.vardrop_probe_bounded_wait(ws, 0)
+
+
+class Guarded:
+    """Buffers cut out of larger allocations whose margins hold a known pattern: any write outside a buffer shows up in a margin."""
+    MARGIN = 4096          # bytes on each side (a multiple of every alignment the library asks for)
+
+    def __init__(self):
+        self.items = []
+
+    def alloc(self, shape, dtype, fill=0):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((n + 2 * self.MARGIN,), 0xA5, dtype=torch.uint8, device="cuda")
+        view = raw[self.MARGIN: self.MARGIN + n].view(dtype).view(shape)
+        view.fill_(fill)
+        self.items.append((raw, n))
+        return view
+
+    def check(self):
+        for raw, n in self.items:
+            assert bool((raw[: self.MARGIN] == 0xA5).all()) and bool((raw[self.MARGIN + n:] == 0xA5).all()), "a margin was written"
+
+
+@pytest.mark.parametrize("name,N", [("elec", None), ("traffic", None), ("scale", 2304)])
+def test_no_write_outside_any_output_or_workspace(name, N):
+    """Every output and every workspace of a whole step sits between guard margins: gathered, staged and many-tile launch shapes
+    (the Scale shape cut to 2304 variates keeps the three-kernel selection and the four-warpgroup attention kernels in play)."""
+    w = inputs.WORKLOADS[name]
+    N = w.N if N is None else N
+    B = min(w.B, 4)
+    x = torch.from_numpy(inputs.make_windows(w, B=B, N=N)).cuda()
+    toks = [torch.from_numpy(t).cuda().to(torch.bfloat16) for t in inputs.make_tokens(B, N, w.H, w.D, w.qkv_std, seed=9)]
+    g = Guarded()
+    hcfg = vd.HashCfg(B, N, w.L, w.k, 0, 0, 0)
+    scfg = vd.SelectCfg(1, N, 0, w.rate, SEED, STEP)
+    acfg = vd.AttnCfg(B, N, w.H, w.D, 0.0)
+    keys = g.alloc((1, N), torch.int64)
+    freqs = g.alloc((1, N, w.k), torch.int32)
+    hws = g.alloc((vd.vardrop_hash_workspace_bytes(hcfg),), torch.uint8)
+    sws = g.alloc((vd.vardrop_select_workspace_bytes(scfg),), torch.uint8)
+    aws = g.alloc((vd.vardrop_attn_workspace_bytes(acfg),), torch.uint8)
+    so = {n_: g.alloc(s_, torch.int32) for n_, s_ in (("group_id", (1, N)), ("group_offsets", (1, N + 1)), ("members", (1, N)), ("n_groups", (1,)),
+                                                       ("sel_idx", (1, N)), ("n_sel", (1,)), ("inv_idx", (1, N)))}
+    o, dq, dk, dv = (g.alloc((B, N, w.H, w.D), torch.bfloat16) for _ in range(4))
+    lse = g.alloc((B, w.H, N), torch.float32)
+    xs = g.alloc((B, N, w.L), torch.float32)
+    vd.vardrop_hash(x, hcfg, keys, freqs, None, hws)
+    vd.vardrop_select(keys, scfg, so["group_id"], so["group_offsets"], so["members"], so["n_groups"], so["sel_idx"], so["n_sel"], so["inv_idx"], sws)
+    vd.vardrop_gather_rows(x, so["sel_idx"], so["n_sel"], vd.GatherCfg(B, N, w.L, 1), xs)
+    vd.vardrop_attn_fwd(toks[0], toks[1], toks[2], so["sel_idx"], so["n_sel"], acfg, o, lse, aws)
+    vd.vardrop_attn_bwd(toks[0], toks[1], toks[2], o, lse, toks[3], so["sel_idx"], so["n_sel"], so["inv_idx"], acfg, dq, dk, dv, aws)
+    vd.vardrop_attn_fwd(toks[0], toks[1], toks[2], None, None, acfg, o, lse, aws)                      # and the all-token kernels
+    vd.vardrop_attn_bwd(toks[0], toks[1], toks[2], o, lse, toks[3], None, None, None, acfg, dq, dk, dv, aws)
+    torch.cuda.synchronize()
+    for ws in (hws, sws, aws):
+        assert vd.ws_status(ws) == vd.OK
+    g.check()
