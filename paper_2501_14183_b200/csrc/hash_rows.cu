@@ -4,14 +4,18 @@
 // Work is laid out by hash row (one variate): a team of 1, 2 or 4 warps owns a row, each warp takes a
 // contiguous range of the batch.  Two real windows ride one complex transform of length L = R1 * R2
 // (z = x_b + i x_{b+1};  X_b[f] = (Z_f + conj Z_{L-f}) / 2,  X_{b+1}[f] = (Z_f - conj Z_{L-f}) / 2i):
-//   pass 1   R2 lanes per transform: lane j2 loads z[j1 R2 + j2] straight from global memory, runs an
+//   staging  the copy engine brings a warp's next windows into shared memory (one bulk copy a window, counted on the warp's
+//            mbarrier) while the warp is in pass 2 of the current ones (x is 16-byte aligned and so is every window),
+//   pass 1   R2 lanes per transform: lane j2 takes z[j1 R2 + j2] from the staged windows, runs an
 //            R1-point DFT in registers, multiplies output k1 by exp(-2 pi i j2 k1 / L) and parks it in the
 //            warp's exchange buffer,
-//   pass 2   R1 lanes per transform: lane k1 reads its R2 values, runs an R2-point DFT in registers; output
-//            k2 is Z[k1 + R1 k2]; only the candidate band and its mirror image are kept,
-//   then     lane fi adds the amplitudes of bin f_lo + fi of the warp's windows in ascending instance order.
-// Warps never wait for each other inside a row (only __syncwarp); the team's partial sums are added in
-// ascending order by its first warp, which ranks the top k bins and packs the hash value.
+//   pass 2   R1 lanes per transform: lane k1 reads its R2 values and runs an R2-point DFT in registers; output k2 is
+//            Z[k1 + R1 k2].  The mirror term Z[L - g] of g = k1 + R1 k2 is output R2 - 1 - k2 of lane R1 - k1 of the same
+//            transform (output (R2 - k2) mod R2 of lane 0 itself when k1 = 0), so one shuffle pair fetches it and the lane
+//            adds both windows' amplitudes of its bins g <= L / 2 to its accumulators: nothing is parked in between.
+// Warps never wait for each other inside a row (only __syncwarp); the transforms that share a warp add their accumulators
+// in ascending order, then the team's partial sums are added in ascending order by its first warp, which ranks the top k
+// bins and packs the hash value.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -205,27 +209,58 @@ struct RowsParams {
 template <int L, int R1, int R2, int PC>
 struct RowsPlan {
     static_assert(R1 * R2 == L, "L = R1 * R2");
+    static_assert(R1 <= 32, "a transform's second pass fits a warp");
+    static constexpr int G2 = 32 / R1;                                      // transforms per second pass of a warp
+    static_assert(PC % G2 == 0, "whole second passes");
     static constexpr int P2 = R2 | 1;                                       // exchange row pitch (complex), odd: pass-2 reads are conflict-free
     static constexpr int PS = R1 * P2 + ((R2 - R1 * P2) % 16 + 16) % 16;    // pitch between transforms: consecutive lanes keep consecutive banks
-    static constexpr int NACC = (L / 2 + 1 + 31) / 32;                      // accumulators per lane (bins lane, lane + 32, ...)
+    static constexpr int K2N = R2 / 2 + 1;                                  // accumulators per lane: bins k1 + R1 k2 <= L / 2
     static constexpr int exch_elems = PC * PS;
-    static size_t smem_bytes(int nf) {
-        return sizeof(float2) * (static_cast<size_t>(L) + kRowsWarps * (exch_elems + static_cast<size_t>(PC) * 2 * nf)) +
-               sizeof(float) * kRowsWarps * NACC * 32;
-    }
+    static constexpr int LP = L + 4;                                        // pitch of a staged window (floats): rows stay 16-byte aligned
+    static constexpr int stage_elems = 2 * PC * LP;                         // a warp's staged windows: first of every pair, then second
+    static constexpr size_t off_exch = sizeof(float2) * L;
+    static_assert(sizeof(float) * K2N * 32 <= sizeof(float2) * exch_elems, "a warp's partial sums fit its exchange buffer");
+    static constexpr size_t off_stage = (off_exch + sizeof(float2) * kRowsWarps * exch_elems + 15) / 16 * 16;
+    static constexpr size_t off_bar = off_stage + sizeof(float) * kRowsWarps * stage_elems;
+    static constexpr size_t smem_bytes() { return off_bar + sizeof(uint64_t) * kRowsWarps; }
+    static_assert(L % 4 == 0 && off_exch % 16 == 0, "staged windows and their copies are 16-byte aligned");
 };
+
+// One window (bytes, a multiple of 16) from global to shared memory by the copy engine; completion is counted on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst_smem)), "l"(src),
+                 "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Ask for `bytes` (a multiple of 16) at the 16-byte aligned address `p` to be brought into L2; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ float sqrt_fast(float v) {                      // square root by the special-function unit (about 1 ulp)
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
 
 template <int L, int R1, int R2, int PC, int MINB>
 __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const RowsParams P) {
     using Plan = RowsPlan<L, R1, R2, PC>;
-    constexpr int P2 = Plan::P2, PS = Plan::PS, NACC = Plan::NACC;
+    constexpr int P2 = Plan::P2, PS = Plan::PS, K2N = Plan::K2N, G2 = Plan::G2, LP = Plan::LP;
     extern __shared__ __align__(16) unsigned char smem_rows[];
     const int nf = P.nf, f_lo = P.f_lo, f_hi = P.f_lo + P.nf;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float2* tw = reinterpret_cast<float2*>(smem_rows);                       // tw[k1 R2 + j2] = exp(-2 pi i j2 k1 / L)
-    float* part = reinterpret_cast<float*>(tw + L);                          // [warps][NACC * 32] partial sums of the team
-    float2* exch = reinterpret_cast<float2*>(part + kRowsWarps * NACC * 32) + static_cast<size_t>(warp) * (Plan::exch_elems + PC * 2 * nf);
-    float2* band = exch + Plan::exch_elems;                                  // [PC][2 nf]: Z_f for the band, then Z_{L-f}
+    float2* exch = reinterpret_cast<float2*>(smem_rows + Plan::off_exch) + static_cast<size_t>(warp) * Plan::exch_elems;
+    // partial sums of a team member, [K2N][32]: they live in the member's own exchange buffer, which is idle between rows
+    auto part_of = [&](int w) { return reinterpret_cast<float*>(smem_rows + Plan::off_exch) + static_cast<size_t>(w) * Plan::exch_elems * 2; };
+    float* stage = reinterpret_cast<float*>(smem_rows + Plan::off_stage) + static_cast<size_t>(warp) * Plan::stage_elems;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_rows + Plan::off_bar) + warp;     // this warp's staged windows have landed
+    if (lane == 0) {
+        mbar_init(bar, 1);
+        mbar_fence_init();
+    }
 
     for (int m = threadIdx.x; m < L; m += kRowsThreads) {
         const int k1 = m / R2, j2 = m - k1 * R2;
@@ -241,32 +276,59 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
 
     const int rows_per_cta = kRowsWarps / P.team;
     const int member = warp % P.team;
-    const float inv_n = 1.f / static_cast<float>(P.B);
+    const float inv_n = 0.5f / static_cast<float>(P.B);                      // the halves of the two-for-one split are taken at the end
+    const int grp = lane / R1, k1 = lane - grp * R1;                         // second pass: transform of the pass, first index
+    const bool lane_used = grp < G2;
+    const int partner = lane_used ? lane - k1 + (R1 - k1) % R1 : lane;       // holds the mirror terms of this lane's outputs
+    const int row_step = gridDim.x * rows_per_cta;
+    const int b_lo = member * P.per_member, b_end = min(P.B, b_lo + P.per_member);     // this warp's windows of a row
+    uint32_t landed = 0;                                                     // parity of the mbarrier phase to wait for next
+    // Stage windows [c, c + 2 PC) of `row` (those below b_end): lane 0 announces the bytes, lane w copies window c + w.
+    auto stage_windows = [&](int row, int c) {
+        const int n = min(2 * PC, b_end - c);
+        // (the warp's reads of the staged windows are complete: their values went through the transform before the
+        // __syncwarp that precedes this call)
+        if (lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(n) * L * sizeof(float));
+        __syncwarp();
+        if (lane < n)
+            bulk_load(stage + ((lane & 1) * PC + (lane >> 1)) * LP, P.x + (static_cast<size_t>(c + lane) * P.N + row) * L, L * sizeof(float), bar);
+    };
+    {
+        const int row0 = blockIdx.x * rows_per_cta + warp / P.team;
+        if (row0 < P.N && b_lo < b_end) stage_windows(row0, b_lo);
+    }
 
     for (int row_base = blockIdx.x * rows_per_cta; row_base < P.N; row_base += gridDim.x * rows_per_cta) {
         const int row = row_base + warp / P.team;
         const bool active = row < P.N;
-        float acc[NACC];
+        float acc[K2N];                                                      // acc[k2]: bin k1 + R1 k2 over this lane's transforms
 #pragma unroll
-        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
+        for (int i = 0; i < K2N; ++i) acc[i] = 0.f;
 
-        const int b_lo = member * P.per_member;
-        const int b_hi = active ? min(P.B, b_lo + P.per_member) : 0;
+        const int b_hi = active ? b_end : 0;
+        // the windows this warp transforms after this row's: ask for them now, so that they wait in L2 by the time they are copied
+        const int next_row = row + row_step;
+        if (next_row < P.N) {
+            for (int b = b_lo + lane; b < b_end; b += 32)
+                prefetch_l2(P.x + (static_cast<size_t>(b) * P.N + next_row) * L, L * sizeof(float));
+        }
         for (int c0 = b_lo; c0 < b_hi; c0 += 2 * PC) {
             const int n_win = min(2 * PC, b_hi - c0);
             const int n_pair = (n_win + 1) >> 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar, landed)) && lane == 0) set_status(P.status, VARDROP_ERR_TIMEOUT);
+            landed ^= 1u;
             // ---- pass 1 ---------------------------------------------------------------------------------------
             for (int t = lane; t < n_pair * R2; t += 32) {
                 const int p = t / R2, j2 = t - p * R2;
                 const int b1 = c0 + 2 * p;
-                const float* s1 = P.x + (static_cast<size_t>(b1) * P.N + row) * L + j2;
                 const bool two = b1 + 1 < b_hi;
-                const float* s2 = s1 + (two ? static_cast<size_t>(P.N) * L : 0);
                 float2 v[R1], y[R1];
+                const float* s1 = stage + p * LP + j2;
+                const float* s2 = s1 + (two ? PC * LP : 0);
                 static_for<0, R1>([&](auto J) {
                     constexpr int j1 = decltype(J)::value;
-                    v[j1].x = __ldg(s1 + j1 * R2);
-                    v[j1].y = __ldg(s2 + j1 * R2);
+                    v[j1].x = s1[j1 * R2];
+                    v[j1].y = s2[j1 * R2];
                 });
                 if (!two) {
                     static_for<0, R1>([&](auto J) { v[decltype(J)::value].y = 0.f; });
@@ -281,70 +343,68 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
                 });
             }
             __syncwarp();
-            // ---- pass 2 ---------------------------------------------------------------------------------------
-            for (int t = lane; t < n_pair * R1; t += 32) {
-                const int p = t / R1, k1 = t - p * R1;
-                const float2* src = exch + p * PS + k1 * P2;
+            // the staged windows are consumed: bring in the next ones
+            if (c0 + 2 * PC < b_hi) stage_windows(row, c0 + 2 * PC);
+            else if (next_row < P.N && b_lo < b_end) stage_windows(next_row, b_lo);
+            // ---- pass 2, amplitudes -------------------------------------------------------------------------------
+            for (int p0 = 0; p0 < n_pair; p0 += G2) {
+                const int p = p0 + grp;
+                const bool live = lane_used && p < n_pair;
+                const float2* src = exch + (live ? p : 0) * PS + (lane_used ? k1 : 0) * P2;
                 float2 v[R2], y[R2];
                 static_for<0, R2>([&](auto J) { v[decltype(J)::value] = src[decltype(J)::value]; });
-                dft<R2, 1, 1>(v, y);
-                float2* bp = band + p * 2 * nf;
-                static_for<0, R2>([&](auto K) {
+                dft<R2, 1, 1>(v, y);                                     // y[k2] = Z[k1 + R1 k2]
+                const bool two = 2 * p + 1 < n_win;
+                static_for<0, K2N>([&](auto K) {
                     constexpr int k2 = decltype(K)::value;
-                    const int g = k1 + R1 * k2;                       // y[k2] = Z_g
-                    const int gm = g == 0 ? 0 : L - g;                // Z_g is the mirror term of bin gm
-                    if (g >= f_lo && g < f_hi) bp[g - f_lo] = y[k2];
-                    if (gm >= f_lo && gm < f_hi) bp[nf + gm - f_lo] = y[k2];
+                    constexpr int far = R2 - 1 - k2, own = (R2 - k2) % R2;
+                    float mx = __shfl_sync(0xffffffffu, y[far].x, partner), my = __shfl_sync(0xffffffffu, y[far].y, partner);
+                    if (k1 == 0) { mx = y[own].x; my = y[own].y; }
+                    const float re1 = y[k2].x + mx, im1 = y[k2].y - my;
+                    const float re2 = y[k2].y + my, im2 = mx - y[k2].x;
+                    const float a1 = sqrt_fast(fmaf(re1, re1, im1 * im1));
+                    const float a2 = sqrt_fast(fmaf(re2, re2, im2 * im2));
+                    if (live) acc[k2] += two ? a1 + a2 : a1;
                 });
             }
             __syncwarp();
-            // ---- amplitudes of the warp's windows, ascending instance order ----------------------------------
+        }
+        // the transforms that shared a second pass: their sums go to the first of them, in ascending order
 #pragma unroll
-            for (int i = 0; i < NACC; ++i) {
-                const int fi = lane + 32 * i;
-                if (fi < nf) {
-                    float a = acc[i];
-                    for (int p = 0; p < n_pair; ++p) {
-                        const float2 z1 = band[p * 2 * nf + fi];
-                        const float2 z2 = band[p * 2 * nf + nf + fi];
-                        const float re1 = z1.x + z2.x, im1 = z1.y - z2.y;
-                        a += 0.5f * sqrtf(fmaf(re1, re1, im1 * im1));
-                        if (2 * p + 1 < n_win) {
-                            const float re2 = z1.y + z2.y, im2 = z2.x - z1.x;
-                            a += 0.5f * sqrtf(fmaf(re2, re2, im2 * im2));
-                        }
-                    }
-                    acc[i] = a;
-                }
+        for (int j = 1; j < G2; ++j) {
+#pragma unroll
+            for (int i = 0; i < K2N; ++i) {
+                const float other = __shfl_sync(0xffffffffu, acc[i], (lane + j * R1) & 31);
+                if (lane < R1) acc[i] += other;
             }
-            __syncwarp();
         }
 
         // ---- team sum in ascending member order ------------------------------------------------------------------
         if (P.team > 1) {
             if (member != 0) {
 #pragma unroll
-                for (int i = 0; i < NACC; ++i) part[(warp * NACC + i) * 32 + lane] = acc[i];
+                for (int i = 0; i < K2N; ++i) part_of(warp)[i * 32 + lane] = acc[i];
             }
             __syncthreads();
             if (member == 0) {
                 for (int m = 1; m < P.team; ++m) {
 #pragma unroll
-                    for (int i = 0; i < NACC; ++i) acc[i] += part[((warp + m) * NACC + i) * 32 + lane];
+                    for (int i = 0; i < K2N; ++i) acc[i] += part_of(warp + m)[i * 32 + lane];
                 }
             }
             __syncthreads();
         }
 
         // ---- top-k ranking (descending amplitude, lower bin first on ties) and packing --------------------------
+        // lane k1 < R1 holds bin k1 + R1 i in acc[i]
         if (active && member == 0) {
             bool bad = false;
 #pragma unroll
-            for (int i = 0; i < NACC; ++i) {
-                const int fi = lane + 32 * i;
-                if (fi < nf) {
+            for (int i = 0; i < K2N; ++i) {
+                const int bin = lane + R1 * i;
+                if (lane < R1 && bin >= f_lo && bin < f_hi) {
                     bad |= !isfinite(acc[i]);
-                    if (P.amp_dbg) P.amp_dbg[static_cast<size_t>(row) * nf + fi] = acc[i] * inv_n;
+                    if (P.amp_dbg) P.amp_dbg[static_cast<size_t>(row) * nf + bin - f_lo] = acc[i] * inv_n;
                 } else {
                     acc[i] = -1.f;                                   // not a candidate
                 }
@@ -352,25 +412,23 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
             if (__any_sync(0xffffffffu, bad) && lane == 0) set_status(P.status, VARDROP_ERR_NONFINITE);
             uint64_t key = 0;
             for (int rank = 0; rank < P.k; ++rank) {
-                // a candidate is coded (amplitude bits, ~bin): amplitudes are non-negative, so unsigned order is
-                // amplitude first, then the lower bin; code 0 = nothing left (taken bins are negative)
-                uint64_t best = 0;
+                // the largest amplitude left, then the lowest bin that has it: two warp-wide integer reductions.  Amplitudes
+                // are non-negative, so their bit patterns order like the values; 0 = nothing left (taken bins are negative).
+                float top = -1.f;
 #pragma unroll
-                for (int i = 0; i < NACC; ++i) {
-                    const uint64_t code = (static_cast<uint64_t>(__float_as_uint(acc[i])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(lane + 32 * i));
-                    if (acc[i] >= 0.f && code > best) best = code;
-                }
+                for (int i = 0; i < K2N; ++i) top = fmaxf(top, acc[i]);
+                const unsigned top_all = __reduce_max_sync(0xffffffffu, top >= 0.f ? __float_as_uint(top) + 1u : 0u);
+                unsigned bin = 0xffffffffu;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    const uint64_t other = __shfl_xor_sync(0xffffffffu, best, off);
-                    best = other > best ? other : best;
-                }
-                const int best_f = best ? static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(best)) : 0;   // 0 only with non-finite input
+                for (int i = K2N - 1; i >= 0; --i)
+                    if (acc[i] >= 0.f && __float_as_uint(acc[i]) + 1u == top_all) bin = static_cast<unsigned>(lane + R1 * i);
+                const unsigned bin_all = __reduce_min_sync(0xffffffffu, bin);
+                const int best_bin = top_all ? static_cast<int>(bin_all) : f_lo;          // f_lo only with non-finite input
 #pragma unroll
-                for (int i = 0; i < NACC; ++i)
-                    if (lane + 32 * i == best_f) acc[i] = -1.f;
-                if (lane == 0 && P.freqs) P.freqs[static_cast<size_t>(row) * P.k + rank] = f_lo + best_f;
-                key = (key << 12) | static_cast<uint64_t>(f_lo + best_f);
+                for (int i = 0; i < K2N; ++i)
+                    if (lane + R1 * i == best_bin) acc[i] = -1.f;
+                if (lane == 0 && P.freqs) P.freqs[static_cast<size_t>(row) * P.k + rank] = best_bin;
+                key = (key << 12) | static_cast<uint64_t>(best_bin);
             }
             if (lane == 0) P.keys[row] = key;
         }
@@ -380,13 +438,13 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
 template <int L, int R1, int R2, int PC, int MINB>
 int launch_rows(const RowsParams& P, cudaStream_t stream) {
     using Plan = RowsPlan<L, R1, R2, PC>;
-    const size_t smem = Plan::smem_bytes(P.nf);
+    const size_t smem = Plan::smem_bytes();
     static thread_local int attr_dev = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (attr_dev != dev) {
         if (int st = check_cuda(cudaFuncSetAttribute(hash_rows_kernel<L, R1, R2, PC, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                     static_cast<int>(Plan::smem_bytes(L / 2 + 1))), "hash: smem attribute"))
+                                                     static_cast<int>(smem)), "hash: smem attribute"))
             return st;
         attr_dev = dev;
     }
@@ -416,11 +474,12 @@ int hash_rows_launch(const float* x, const vardrop_hash_cfg& c, int f_lo, int f_
     int team = 1;
     while (team < kRowsWarps && static_cast<long long>(c.N) * team < 8ll * sm_count() && c.B >= 8 * team) team *= 2;
     P.team = team;
+    if (reinterpret_cast<uintptr_t>(x) % 16 != 0) return fail(VARDROP_ERR_INVALID_ARG, "hash: x is not 16-byte aligned");
     int per = (c.B + team - 1) / team;
     P.per_member = per + (per & 1);
     switch (c.L) {
-        case 96: return launch_rows<96, 8, 12, 8, 5>(P, stream);
-        case 192: return launch_rows<192, 12, 16, 4, 3>(P, stream);
+        case 96: return launch_rows<96, 8, 12, 4, 5>(P, stream);
+        case 192: return launch_rows<192, 12, 16, 2, 3>(P, stream);
         case 336: return launch_rows<336, 16, 21, 2, 4>(P, stream);
         default: return launch_rows<720, 24, 30, 1, 4>(P, stream);
     }

@@ -76,6 +76,29 @@ def test_select_long_rows():
     assert got["n_groups"][0] == 4096 and got["n_sel"][0] == 4096
 
 
+def test_select_middle_rows():
+    """Rows of 2049 .. 8192 variates: ragged sizes, keys that differ in all 64 bits or in a single one, one group, two groups
+    of very different size, many equal groups of 512, 20 and 2 members, several rows at once."""
+    rng = np.random.default_rng(5)
+    wide = rng.integers(0, 2**63, size=5000, dtype=np.uint64) * np.uint64(2) + rng.integers(0, 2, size=5000, dtype=np.uint64)
+    wide[rng.integers(0, 5000, size=700)] = wide[0]                        # one longer group among distinct keys
+    wide[1] = np.uint64(0xFFFFFFFFFFFFFFFF)
+    wide[2] = np.uint64(0)
+    check(wide, 10, 1.0, seed=12, step=3)
+    check(wide, 0, 0.3, seed=12, step=4)
+    one_bit = (rng.integers(0, 2, size=8191, dtype=np.uint64) << np.uint64(63)) | np.uint64(0x123)
+    got = check(one_bit, 0, 0.01, seed=2, step=0)
+    assert got["n_groups"][0] == 2
+    for N in (2049, 3073, 8191, 8192):
+        for sizes in ([N], [N - 1, 1], [512] * (N // 512) + [N % 512], [20] * (N // 20) + [N % 20], [2] * (N // 2) + [N % 2]):
+            sizes = [n for n in sizes if n > 0]
+            keys = np.concatenate([np.full(n, (i * 0x9E3779B97F4A7C15) % 2**48, dtype=np.uint64) for i, n in enumerate(sizes)])
+            keys = keys[rng.permutation(len(keys))]
+            check(keys, 7, 0.4, seed=N, step=len(sizes) % 5)
+    rows = np.stack([inputs.make_keys(6000, 10 + 700 * s, k=5, f_hi=361, seed=60 + s) for s in range(4)])
+    check(rows, 0, 0.1, seed=31, step=2)
+
+
 def test_select_random_configurations():
     """Seeded random draws of (N, rows, groups, gs, rate, k) on both sides of every size limit of the kernels
     (2048: one-CTA path; 18432: grouping in shared memory; 65536: the largest N)."""
