@@ -185,6 +185,37 @@ __device__ __forceinline__ void store_chunk16(unsigned char* tile, int r, int c0
     }
 }
 
+// Zero rows of dq, dk, dv for every dropped variate, by one warp of the CTA that is off the critical path, so that the zeros
+// are written beside the products instead of in front of them.  The rows of all instances are dealt to the CTAs in rounds of
+// 32: in round k the warp of CTA c looks rows (c + k gridDim.x) 32 .. + 31 up in inv_idx, one a lane, and writes the dropped
+// ones, 512 bytes a store instruction.
+__device__ __forceinline__ int zero_row_rounds(const BwdParams& P) {
+    return P.inv_idx ? (P.B * P.N + static_cast<int>(gridDim.x) * 32 - 1) / (static_cast<int>(gridDim.x) * 32) : 0;
+}
+__device__ __forceinline__ void zero_rows_round(const BwdParams& P, int round) {
+    const int lane = threadIdx.x & 31;
+    const int chunks_row = P.H * (P.D / 8);                    // 16-byte chunks per (instance, variate) row
+    const int total_rows = P.B * P.N;
+    const int base = (static_cast<int>(blockIdx.x) + round * static_cast<int>(gridDim.x)) * 32;
+    const int r = base + lane;
+    bool dropped = false;
+    if (r < total_rows) {
+        const int b = r / P.N, n = r - b * P.N;
+        dropped = __ldg(P.inv_idx + static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n) < 0;
+    }
+    unsigned mask = __ballot_sync(0xffffffffu, dropped);
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
+    uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
+    uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
+    while (mask) {
+        const int l = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
+        for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
+    }
+}
+
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                    const __grid_constant__ CUtensorMap map_k,
                                                                    const __grid_constant__ CUtensorMap map_v,
@@ -259,37 +290,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const int kept_shared = P.n_sel ? (P.S > 1 ? -1 : __ldg(P.n_sel)) : P.N;
     const int n_t_max = ((P.S > 1 ? max_kept(P.n_sel, P.S, P.N, reinterpret_cast<int*>(smem_dyn + 100)) : kept_shared) + kTile - 1) / kTile;     // tiles of the longest selection
     const int n_items = n_t_max * P.H * P.B;                   // work items: (key tile, head, instance); short instances skip tiles
-    // Zero rows of dq, dk, dv for every dropped variate, spread over the warps of the whole grid.  Each CTA runs it once, behind the
-    // operand loads of its first work item, so the stores drain while those loads are in flight.
-    bool zeros_written = P.inv_idx == nullptr;
-    auto write_zero_rows = [&]() {
-        zeros_written = true;
-        const int chunks_row = P.H * (P.D / 8);                // 16-byte chunks per (instance, variate) row
-        const int total_rows = P.B * P.N;
-        const int lane = threadIdx.x & 31;
-        const int warps_grid = gridDim.x * (kBwdWorkers >> 5);
-        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
-        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
-        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
-        int group = 1;                                         // rows looked up per warp and round: enough to give every warp work, at most 32
-        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
-        for (int base = (blockIdx.x * (kBwdWorkers >> 5) + (threadIdx.x >> 5)) * group; base < total_rows; base += warps_grid * group) {
-            const int r = base + lane;                         // lanes 0 .. group-1 look up one row each, then the warp writes the dropped ones
-            bool dropped = false;
-            if (lane < group && r < total_rows) {
-                const int b = r / P.N, n = r - b * P.N;
-                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, dropped);
-            while (mask) {
-                const int l = __ffs(mask) - 1;
-                mask &= mask - 1;
-                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
-                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
-            }
-        }
-    };
+    // Zero rows of dq, dk, dv for every dropped variate: the last warp of the third warpgroup, which only helps with taking dQ out
+    // of tensor memory, writes a slice of its CTA's share ahead of every query tile (see zero_rows_round) and the rest at the end.
+    const bool zero_warp = warp == kBwdThreads / 32 - 1 && P.inv_idx != nullptr;
     // (a CTA past the last item runs no loop below: it writes its share of the zero rows and frees its tensor memory)
 
     const uint32_t tm_st = tmem;            // [0,128)   S^T
@@ -387,6 +390,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         // tile out of tensor memory into the fp32 shared-memory tile, which one bulk reduction adds to the accumulator.
         const bool issuer = tid == kBwdWorkers;
         const int qrow_l = tid - kBwdWorkers;           // query row this thread drains
+        const int z_rounds = zero_warp ? zero_row_rounds(P) : 0;
+        const int tiles_cta = (n_items > static_cast<int>(blockIdx.x) ? (n_items - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0) * n_t_max;
+        const int z_slice = tiles_cta > 0 ? (z_rounds + tiles_cta - 1) / tiles_cta : z_rounds;      // rounds ahead of every query tile
+        int z_round = 0;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int jt = item % n_t_max;
             const int h = (item / n_t_max) % P.H;
@@ -405,6 +412,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             }
             for (int i = 0; i < n_q; ++i) {
                 const uint32_t qc = q_count + i, st = qc % kQStages, st1 = (qc + 1) % kQStages, ph = qc & 1;
+                for (int zs = 0; zs < z_slice && z_round < z_rounds; ++zs, ++z_round) zero_rows_round(P, z_round);
                 if (issuer) {
                     ok &= mbar_wait(bar_p, ph);
                     tc_fence_after();
@@ -462,9 +470,32 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             q_count += n_q;
             ++n_done;
         }
+        for (; z_round < z_rounds; ++z_round) zero_rows_round(P, z_round);    // what is left of the zero rows
         if (tid == kBwdWorkers) bulk_wait_group0();      // the last dQ reductions have landed
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kBwdWorkerRegs));
+    // Operand fetches of a work item: K, V and the first two query tiles' Q, dO, by warps 0 .. 3 side by side (each looks up its own
+    // gather rows); a barrier phase cannot complete before the thread that announces its bytes has arrived, whichever comes
+    // first.  `qc` is the number of query tiles this CTA has consumed before the item (its first ring stage).
+    auto fetch_item = [&](int jt_, int h_, int b_, int kept_, uint32_t qc) {
+        const int srow_ = P.S > 1 ? b_ : 0;
+        TileSource src_ = P.src, src_do_ = P.src_do;
+        if (src_.idx) src_.idx += static_cast<size_t>(srow_) * P.N;
+        const int n_q_ = (kept_ + kTile - 1) / kTile;
+        if (tid == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
+        if (warp == 0) load_tile(sK, &map_k, bar_kv, src_, jt_ * kTile, kept_, h_, b_, P.H);
+        else if (warp == 1) load_tile(sV, &map_v, bar_kv, src_, jt_ * kTile, kept_, h_, b_, P.H);
+        for (int i = 0; i < 2 && i < n_q_; ++i) {
+            const uint32_t stage = (qc + i) % kQStages;
+            if (warp == 2) {
+                if ((tid & 31) == 0) mbar_expect_tx(bar_qdo + stage, 2 * kTileBytes);
+                load_tile(sQ + stage * kTileBytes, &map_q, bar_qdo + stage, src_, i * kTile, kept_, h_, b_, P.H);
+            } else if (warp == 3) {
+                load_tile(sdO + stage * kTileBytes, &map_do, bar_qdo + stage, src_do_, i * kTile, kept_, h_, b_, P.H);
+            }
+        }
+    };
+    bool fetched = false;       // the operands of the item at hand were requested behind the products of the item before it
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const int jt = item % n_t_max;
         const int h = (item / n_t_max) % P.H;
@@ -499,21 +530,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         float dl_cur = load_delta(b, h, row), dl_next = 0.f;
         if (!use_delta) load_o(b, h, row, o_cur);
         const int n_out = key_valid ? (sel ? sel[key] : key) : 0;
-        {   // every MMA of the previous item has completed: K, V and every Q/dO stage are free.  Warps 0 .. 3 fetch K, V, Q, dO
-            // side by side (each looks up its own gather rows); a barrier phase cannot complete before the thread that
-            // announces its bytes has arrived, whichever comes first.
-            if (tid == 0) mbar_expect_tx(bar_kv, 2 * kTileBytes);
-            if (warp == 0) load_tile(sK, &map_k, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            else if (warp == 1) load_tile(sV, &map_v, bar_kv, src, jt * kTile, n_sel, h, b, P.H);
-            fetch_qdo(0, st0);
-            if (n_q > 1) fetch_qdo(1, (st0 + 1) % kQStages);
-        }
+        if (!fetched) fetch_item(jt, h, b, n_sel, q_count);      // (the CTA's first item: nothing came before it)
+        fetched = false;
         if (half == 0) {
             s_stat[st0 * kTile + row] = lse_first;
             if (n_q > 1) s_stat[((st0 + 1) % kQStages) * kTile + row] = lse_second;
         }
         if (use_delta && half == 1) s_dpart[(q_count & 1) * kTile + row] = dl_cur;      // Delta of the first tile, in its parity's array
-        if (!zeros_written) write_zero_rows();
         worker_sync();                                   // row statistics of the first tiles visible
 
         // The query loop is a two-phase pipeline.  Phase A turns S^T into P^T while the tensor core still runs dK, dP^T of the
@@ -629,6 +652,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 
         ok &= mbar_wait(bar_acc, n_done & 1);
         tc_fence_after();
+        // Every product of this item has completed: K, V and every Q / dO stage are free, and nothing below touches them.  The
+        // operands of this CTA's next item are requested now, so that they travel while the gradients of this one are written;
+        // the issuing thread then queues that item's first S^T and dP^T (tensor-memory columns the write-out does not read).
+        if (ok) {
+            for (int nx = item + gridDim.x; nx < n_items; nx += gridDim.x) {
+                const int jt_n = nx % n_t_max, h_n = (nx / n_t_max) % P.H, b_n = nx / (n_t_max * P.H);
+                const int kept_n = P.S > 1 ? P.n_sel[b_n] : kept_shared;
+                if (jt_n >= (kept_n + kTile - 1) / kTile) continue;
+                fetch_item(jt_n, h_n, b_n, kept_n, q_count);
+                fetched = true;
+                break;
+            }
+        }
         {   // dV, dK of this key tile (and dQ when this is the only key tile: key row = query row): every thread rounds its 32
             // columns to bf16 into a staging tile (the P^T / dS^T tiles are free now), then eight threads write each 128-byte
             // row of the full-layout gradients in one piece.
@@ -689,7 +725,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         ++n_done;
     }
     }   // workers
-    if (!zeros_written && tid < kBwdWorkers) write_zero_rows();           // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();
@@ -829,37 +864,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
         it.n_q = (it.n_sel + kTile - 1) / kTile;               // query tiles = key tiles of this instance
         return it;
     };
-    // zero rows of dq, dk, dv for every dropped variate, spread over the 16 phase warps of the whole grid; each CTA runs it once
-    bool zeros_written = P.inv_idx == nullptr;
-    auto write_zero_rows = [&]() {
-        zeros_written = true;
-        const int chunks_row = P.H * (P.D / 8);
-        const int total_rows = P.B * P.N;
-        const int lane = threadIdx.x & 31;
-        const int warps_cta = 2 * kPipeGroup / 32;
-        const int warps_grid = gridDim.x * warps_cta;
-        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-        uint4* dq4 = reinterpret_cast<uint4*>(P.dq);
-        uint4* dk4 = reinterpret_cast<uint4*>(P.dk);
-        uint4* dv4 = reinterpret_cast<uint4*>(P.dv);
-        int group = 1;
-        while (group < 32 && group * warps_grid < total_rows) group <<= 1;
-        for (int base = (blockIdx.x * warps_cta + (warp - 4)) * group; base < total_rows; base += warps_grid * group) {
-            const int r = base + lane;
-            bool dropped = false;
-            if (lane < group && r < total_rows) {
-                const int b = r / P.N, n = r - b * P.N;
-                dropped = P.inv_idx[static_cast<size_t>(P.S > 1 ? b : 0) * P.N + n] < 0;
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, dropped);
-            while (mask) {
-                const int l = __ffs(mask) - 1;
-                mask &= mask - 1;
-                const size_t row0 = static_cast<size_t>(base + l) * chunks_row;
-                for (int c = lane; c < chunks_row; c += 32) { dq4[row0 + c] = z; dk4[row0 + c] = z; dv4[row0 + c] = z; }
-            }
-        }
-    };
     // bf16 staging of a 64-column accumulator (this thread's 32 columns of its key row), then whole 128-byte rows to the
     // full-layout gradient: used by phase A for dV and by phase B for dK (and dQ of a single-tile instance)
     auto stage_acc = [&](unsigned char* tile, uint32_t tm, float mul, int row, int half) {
@@ -887,6 +891,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
     if (warp < 4) {
         // ------------------------------------------------------------ issue and dQ drain --------------------------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPipeSmallRegs));
+        // the fourth warp of this group issues nothing: it writes the zero rows of the dropped variates
+        if (warp == 3) {
+            const int z_rounds = zero_row_rounds(P);
+            for (int z_round = 0; z_round < z_rounds; ++z_round) zero_rows_round(P, z_round);
+        }
         constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);     // K-major x K-major, N = 128
         constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major (tensor memory), B MN-major, N = 64
         constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
@@ -1021,7 +1030,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
                 s_stat[st0 * kTile + row] = load_lse(row);
                 if (it.n_q > 1) s_stat[((st0 + 1) % kQStages) * kTile + row] = load_lse(kTile + row);
             }
-            if (!zeros_written) write_zero_rows();
             ok = group_sync_and<1>(ok);                  // row statistics of the first tiles visible
             for (int i = 0; i < it.n_q; ++i, ++q_count) {
                 const uint32_t st = q_count % kQStages, ph = q_count & 1, st2 = (q_count + 2) % kQStages;
@@ -1129,7 +1137,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
             }
             if (half == 1) s_delta[(q_count & 1) * kTile + row] = dl_first;
             else s_nout[(n_done & 1) * kTile + row] = n_out;     // phase A reads it at the end of the item; the array of two items ago is free
-            if (!zeros_written) write_zero_rows();
             ok = group_sync_and<3>(ok);
             for (int i = 0; i < it.n_q; ++i, ++q_count) {
                 const uint32_t ph = q_count & 1, st2 = (q_count + 2) % kQStages;
@@ -1199,7 +1206,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
             ++n_done;
         }
     }
-    if (!zeros_written && warp >= 4) write_zero_rows();          // every item of this CTA was skipped (short instances)
     if (!ok) set_status(P.status, VARDROP_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();
