@@ -891,11 +891,6 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
     if (warp < 4) {
         // ------------------------------------------------------------ issue and dQ drain --------------------------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPipeSmallRegs));
-        // the fourth warp of this group issues nothing: it writes the zero rows of the dropped variates
-        if (warp == 3) {
-            const int z_rounds = zero_row_rounds(P);
-            for (int z_round = 0; z_round < z_rounds; ++z_round) zero_rows_round(P, z_round);
-        }
         constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);     // K-major x K-major, N = 128
         constexpr uint32_t idesc_kmn = umma_idesc_bf16(128, kDP, 0, 1);    // A K-major (tensor memory), B MN-major, N = 64
         constexpr uint32_t idesc_mnmn = umma_idesc_bf16(128, kDP, 1, 1);   // A MN-major, B MN-major, N = 64
@@ -988,6 +983,12 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_bwd_pipe_kernel(const __
             if (!ok) break;
             q_count += it.n_q;
             ++n_done;
+        }
+        // The fourth warp of this group issues nothing and falls through the loop above at once: it writes the zero rows of the
+        // dropped variates while the others work.  (Placed behind the loop, this code shares no live range with the issue code.)
+        if (warp == 3) {
+            const int z_rounds = zero_row_rounds(P);
+            for (int z_round = 0; z_round < z_rounds; ++z_round) zero_rows_round(P, z_round);
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------ phase A: P^T --------------------------------------
