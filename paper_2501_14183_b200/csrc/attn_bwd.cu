@@ -104,9 +104,10 @@ constexpr int kBwdWorkers = 256;       // two threads per tensor-memory lane: ea
 constexpr int kBwdThreads = kBwdWorkers + 128; // plus a third warpgroup: its first warp's first lane issues every tensor-core product,
                                                // the rest of it only gives its registers to the workers
 // Register split (setmaxnreg works on whole warpgroups): the kernel is launched with 384 x 168 = 64512 registers; the
-// third warpgroup keeps 136 a thread and the two worker warpgroups take 184: 256 x 184 + 128 x 136 = 64512.
-constexpr int kBwdWorkerRegs = 184;
-constexpr int kBwdIssuerRegs = 136;
+// third warpgroup keeps 152 a thread and the two worker warpgroups take 176: 256 x 176 + 128 x 152 = 64512 (with less than
+// 152 the third warpgroup, which also takes dQ out of tensor memory, spills).
+constexpr int kBwdWorkerRegs = 176;
+constexpr int kBwdIssuerRegs = 152;
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr int kQStages = 3;            // ring of query-tile operands (Q and dO), fetched two tiles ahead
 constexpr int kBwdSmemBytes = 3072 /*barriers, row statistics, alignment*/ + 2 * kTileBytes /*K, V*/ + 2 * kQStages * kTileBytes /*Q, dO ring*/ +
