@@ -8,8 +8,8 @@
 //                    memory; P^T and dS^T are written to shared memory once and feed three tensor-core products:
 //                    dV += P^T dO, dK += dS^T Q (accumulated in tensor memory across the query loop) and
 //                    dQ_i = dS K (added into the fp32 accumulator by bulk reduce-adds).
-//                    The same kernel writes the zero rows of every dropped variate (while its first tiles are in
-//                    flight) and, when the CTA that finishes the last key tile of an (instance, head) pair sees the
+//                    The same kernel writes the zero rows of every dropped variate (by a warp that is off the critical
+//                    path, a slice ahead of every query tile) and, when the CTA that finishes the last key tile of an (instance, head) pair sees the
 //                    pair complete, converts that pair's dQ' accumulator to bf16 rows of dq: each row of dq / dk / dv
 //                    is written exactly once and no further launch is needed.
 #include "attn_common.cuh"
