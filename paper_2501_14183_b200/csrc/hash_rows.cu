@@ -214,7 +214,8 @@ struct RowsPlan {
     static_assert(PC % G2 == 0, "whole second passes");
     static constexpr int P2 = R2 | 1;                                       // exchange row pitch (complex), odd: pass-2 reads are conflict-free
     static constexpr int PS = R1 * P2 + ((R2 - R1 * P2) % 16 + 16) % 16;    // pitch between transforms: consecutive lanes keep consecutive banks
-    static constexpr int K2N = R2 / 2 + 1;                                  // accumulators per lane: bins k1 + R1 k2 <= L / 2
+    static constexpr int K2N = R2 / 2 + 1;                                  // accumulators per lane for the whole spectrum: bins k1 + R1 k2 <= L / 2
+    static constexpr int K2Q = ((L / 2 + 2) / 2 + R1 - 1) / R1;             // for the default band, f < ceil((L / 2 + 1) / 2): bins below R1 K2Q
     static constexpr int exch_elems = PC * PS;
     static constexpr int LP = L + 4;                                        // pitch of a staged window (floats): rows stay 16-byte aligned
     static constexpr int stage_elems = 2 * PC * LP;                         // a warp's staged windows: first of every pair, then second
@@ -244,10 +245,13 @@ __device__ __forceinline__ float sqrt_fast(float v) {                      // sq
     return r;
 }
 
-template <int L, int R1, int R2, int PC, int MINB>
+// kWide: candidate bins may lie anywhere up to L / 2; otherwise the band ends below R1 K2Q (the default low-pass band does), and
+// a lane evaluates, adds up and ranks only its K2Q lowest bins: the outputs of the second pass that no such bin or mirror term
+// reads are never computed.
+template <int L, int R1, int R2, int PC, int MINB, bool kWide>
 __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const RowsParams P) {
     using Plan = RowsPlan<L, R1, R2, PC>;
-    constexpr int P2 = Plan::P2, PS = Plan::PS, K2N = Plan::K2N, G2 = Plan::G2, LP = Plan::LP;
+    constexpr int P2 = Plan::P2, PS = Plan::PS, K2N = kWide ? Plan::K2N : Plan::K2Q, G2 = Plan::G2, LP = Plan::LP;
     extern __shared__ __align__(16) unsigned char smem_rows[];
     const int nf = P.nf, f_lo = P.f_lo, f_hi = P.f_lo + P.nf;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -435,7 +439,7 @@ __global__ void __launch_bounds__(kRowsThreads, MINB) hash_rows_kernel(const Row
     }
 }
 
-template <int L, int R1, int R2, int PC, int MINB>
+template <int L, int R1, int R2, int PC, int MINB, bool kWide>
 int launch_rows(const RowsParams& P, cudaStream_t stream) {
     using Plan = RowsPlan<L, R1, R2, PC>;
     const size_t smem = Plan::smem_bytes();
@@ -443,7 +447,7 @@ int launch_rows(const RowsParams& P, cudaStream_t stream) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (attr_dev != dev) {
-        if (int st = check_cuda(cudaFuncSetAttribute(hash_rows_kernel<L, R1, R2, PC, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (int st = check_cuda(cudaFuncSetAttribute(hash_rows_kernel<L, R1, R2, PC, MINB, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      static_cast<int>(smem)), "hash: smem attribute"))
             return st;
         attr_dev = dev;
@@ -456,7 +460,7 @@ int launch_rows(const RowsParams& P, cudaStream_t stream) {
     const int cap = sm_count() * per_sm;
     const int grid = want < cap ? want : cap;
     cudaError_t err;
-    { LaunchScope ls_(K_HASH, stream); err = launch_chained(hash_rows_kernel<L, R1, R2, PC, MINB>, dim3(grid), dim3(kRowsThreads), smem, stream, P); }
+    { LaunchScope ls_(K_HASH, stream); err = launch_chained(hash_rows_kernel<L, R1, R2, PC, MINB, kWide>, dim3(grid), dim3(kRowsThreads), smem, stream, P); }
     return check_cuda(err, "hash: launch");
 }
 
@@ -478,10 +482,10 @@ int hash_rows_launch(const float* x, const vardrop_hash_cfg& c, int f_lo, int f_
     int per = (c.B + team - 1) / team;
     P.per_member = per + (per & 1);
     switch (c.L) {
-        case 96: return launch_rows<96, 8, 12, 4, 5>(P, stream);
-        case 192: return launch_rows<192, 12, 16, 2, 3>(P, stream);
-        case 336: return launch_rows<336, 16, 21, 2, 4>(P, stream);
-        default: return launch_rows<720, 24, 30, 1, 4>(P, stream);
+        case 96: return f_hi <= 8 * RowsPlan<96, 8, 12, 4>::K2Q ? launch_rows<96, 8, 12, 4, 5, false>(P, stream) : launch_rows<96, 8, 12, 4, 5, true>(P, stream);
+        case 192: return f_hi <= 12 * RowsPlan<192, 12, 16, 2>::K2Q ? launch_rows<192, 12, 16, 2, 3, false>(P, stream) : launch_rows<192, 12, 16, 2, 3, true>(P, stream);
+        case 336: return f_hi <= 16 * RowsPlan<336, 16, 21, 2>::K2Q ? launch_rows<336, 16, 21, 2, 4, false>(P, stream) : launch_rows<336, 16, 21, 2, 4, true>(P, stream);
+        default: return f_hi <= 24 * RowsPlan<720, 24, 30, 1>::K2Q ? launch_rows<720, 24, 30, 1, 4, false>(P, stream) : launch_rows<720, 24, 30, 1, 4, true>(P, stream);
     }
 }
 
