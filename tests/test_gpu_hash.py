@@ -121,6 +121,20 @@ def test_hash_band_options_and_debug_outputs_optional():
     assert np.array_equal(keys_t.cpu().numpy().view(np.uint64), keys)
 
 
+@pytest.mark.parametrize("L,edge", [(96, 32), (192, 60), (336, 96), (720, 192)])
+def test_hash_band_edges_of_the_register_blocked_kernel(L, edge):
+    """The register-blocked kernel has a form for bands that end at or below `edge` bins (a lane then evaluates only its lowest
+    bins) and one for wider bands: bands on both sides of the switch, and the widest one, against the oracle."""
+    nb = L // 2 + 1
+    x = random_periodic(6, 40, L, 3, seed=L)
+    for f_lo, f_hi in [(1, edge - 1), (0, edge), (1, edge + 1), (2, nb)]:
+        xf, keys, freqs, abar, _ = gap_filtered_windows(x, 3, f_lo, f_hi)
+        gk, gf, ga = run_hash(xf, 3, f_lo, f_hi)
+        assert np.array_equal(gf, freqs), (L, f_lo, f_hi)
+        assert np.array_equal(gk, keys), (L, f_lo, f_hi)
+        np.testing.assert_allclose(ga, abar, rtol=2e-5, atol=2e-5 * abar.max())
+
+
 def test_hash_is_deterministic():
     w = inputs.WORKLOADS["elec"]
     x = inputs.make_windows(w)
